@@ -1,0 +1,331 @@
+#!/usr/bin/env python
+"""Throughput of the speculative-prefill scoring + selection path on synthetic long-context prompts.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One step = one pass of the whole path (score -> chunk pool -> top-k -> span compaction) over one batch
+of the workload, inputs resident in HBM.  Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every
+rank runs the same workload shape on its own prompts: prompts are independent, so there is no
+collective on the data path and the scaling is weak.
+
+`--impl reference` times the CPU oracle (plain NumPy fp64, as it stands) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "prompt tokens scored+selected per second"
+UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "long128k"          # N = 131072, the configuration the metric is quoted on
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------------------------- oracle leg
+def oracle_sample(cfg, prompt, keep, sample_layers):
+    """Times the oracle on `sample_layers` of the prompt's layers (all keys) plus the full selection and
+    scales the scoring time to all layers.  Returns (tokens/s, seconds of CPU work, description)."""
+    import numpy as np
+    import oracle
+    from workloads import bf16_bits
+
+    q = bf16_bits(prompt.q[:sample_layers])
+    k = [bf16_bits(x) for x in prompt.k[:sample_layers]]
+    ids, cs, ce = (t.cpu().numpy() for t in (prompt.token_ids, prompt.char_start, prompt.char_end))
+    t0 = time.perf_counter()
+    imp, _ = oracle.token_importance(q, k)
+    t1 = time.perf_counter()
+    scores = oracle.chunk_means(oracle.avg_pool(imp, cfg.pool_kernel), cfg.chunk)
+    kept = oracle.select_topk(scores, oracle.keep_count(len(scores), keep))
+    oracle.compact(kept, cfg.chunk, prompt.n_tokens, ids, cs, ce)
+    t2 = time.perf_counter()
+    t_full = (t1 - t0) * cfg.n_layers / sample_layers + (t2 - t1)
+    desc = (f"oracle on layers 0..{sample_layers - 1} of {cfg.n_layers} (all {prompt.n_tokens} keys, all heads), "
+            f"scoring time scaled x{cfg.n_layers / sample_layers:g}, plus the full selection")
+    return prompt.n_tokens / t_full, t2 - t0, desc
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from workloads import CONFIGS, make_prompt
+    cfg = CONFIGS[args.workload]
+    prompt = make_prompt(cfg, 0, "cuda" if torch.cuda.is_available() else "cpu").to("cpu")
+    keep = cfg.keep[0]
+    sample_layers = 1
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample(cfg, prompt, keep, sample_layers)
+    vals, secs, desc = [], 0.0, ""
+    for _ in range(args.steps):
+        v, s, desc = oracle_sample(cfg, prompt, keep, sample_layers)
+        vals.append(v)
+        secs += s
+    value = len(vals) / sum(1.0 / v for v in vals)
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * cfg.lengths[0] / value, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "n_tokens": cfg.lengths[0], "n_layers": cfg.n_layers,
+                   "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
+                   "n_lookahead": cfg.n_lookahead, "chunk": cfg.chunk, "keep": keep},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2603_02631_b200 as spf
+    from workloads import CONFIGS, make_prompt
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    cfg = CONFIGS[args.workload]
+    keep = cfg.keep[0]
+    n_prompts = len(cfg.lengths)
+    # weak scaling: every rank gets the same shapes, its own prompts (distinct seeds via the prompt index)
+    prompts = [make_prompt(cfg, i, dev) if rank == 0 else
+               make_prompt(__import__("dataclasses").replace(cfg, seed=cfg.seed + 1000 * rank), i, dev)
+               for i in range(n_prompts)]
+    max_n = max(cfg.lengths)
+    sel = spf.Selector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, max_n,
+                       chunk=cfg.chunk, pool_kernel=cfg.pool_kernel, device=dev)
+    tokens_per_step = sum(cfg.lengths)
+    stream = torch.cuda.current_stream()
+    launches_per_prompt = 7      # pack_q, score_lse, merge_lse, score_max, chunk_pool, select_topk, compact_spans
+
+    def step():
+        for p in prompts:
+            sel.run(p.q, p.k, p.token_ids, p.char_start, p.char_end, keep)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # --- device-resident throughput ------------------------------------------------------------
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_start.record(stream)
+    for _ in range(args.steps):
+        step()
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = t_start.elapsed_time(t_end)
+
+    # --- the scoring call on its own (same launches, events around spf_score only) --------------------
+    score_ms = []
+    bufs = [spf.binding.PromptBuffers(p.q, p.k, sel.importance[:p.n_tokens], sel.lse) for p in prompts]
+    ws = sel._workspace(bufs[cfg.lengths.index(max_n)])
+    for it in range(args.steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for bf in bufs:
+            spf.spf_score([bf], ws, 0.0, sel.dev_status)
+        b.record(stream)
+        b.synchronize()
+        score_ms.append(a.elapsed_time(b))
+    score_ms_avg = sum(score_ms) / len(score_ms)
+
+    # --- end to end from pinned host memory -----------------------------------------------------
+    e2e = None
+    if args.e2e_steps > 0:
+        host = []
+        h2d = 0
+        for p in prompts:
+            hp = dict(q=p.q.cpu().pin_memory(), k=[x.cpu().pin_memory() for x in p.k],
+                      ids=p.token_ids.cpu().pin_memory(), cs=p.char_start.cpu().pin_memory(),
+                      ce=p.char_end.cpu().pin_memory())
+            h2d += hp["q"].numel() * 2 + sum(x.numel() * 2 for x in hp["k"]) + 3 * 4 * p.n_tokens
+            host.append(hp)
+        del prompts, bufs
+        torch.cuda.empty_cache()
+
+        def e2e_step():
+            d2h = 0
+            for hp in host:
+                out = sel.run_host(hp["q"], hp["k"], hp["ids"], hp["cs"], hp["ce"], keep)
+                d2h += 16 + sum(v.nbytes for v in out.values())
+            return d2h
+
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        d2h = 0
+        for _ in range(args.e2e_steps):
+            d2h = e2e_step()
+        barrier()
+        e2e_s = time.perf_counter() - t0
+        e2e = {"seconds": e2e_s, "h2d": h2d, "d2h": d2h}
+
+    # --- reduce over ranks --------------------------------------------------------------------------
+    if world > 1:
+        t = torch.tensor([ms_total, e2e["seconds"] if e2e else 0.0, score_ms_avg], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, e2e_s_max, score_ms_avg = t.tolist()
+        if e2e:
+            e2e["seconds"] = e2e_s_max
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    value = world * tokens_per_step * args.steps / (ms_total * 1e-3)
+    peak, peak_kind = hbm_peak()
+    k_bytes = cfg.k_bytes()
+    q_bytes = n_prompts * cfg.n_layers * cfg.n_q_heads * cfg.n_lookahead * cfg.head_dim * 2
+    score_bytes = k_bytes + q_bytes + 4 * tokens_per_step + n_prompts * cfg.n_layers * cfg.n_q_heads * cfg.n_lookahead * 4
+    achieved = score_bytes / (score_ms_avg * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate/softmax", "data": "synthetic",
+        "config": {"workload": cfg.name, "n_prompts_per_gpu": n_prompts, "n_tokens": list(cfg.lengths),
+                   "n_layers": cfg.n_layers, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
+                   "head_dim": cfg.head_dim, "n_lookahead": cfg.n_lookahead, "chunk": cfg.chunk, "keep": keep,
+                   "pool_kernel": cfg.pool_kernel, "k_cache_bytes": k_bytes,
+                   "l2": "inputs larger than L2 (key cache streamed every step)", "parallelism": f"prompts x{world}"},
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "gpu_launches": launches_per_prompt * n_prompts * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "spf_score (pack_q + score_lse + merge_lse + score_max)",
+                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "ms_per_launch": score_ms_avg,
+                     "algorithmic_bytes": score_bytes},
+    }
+    if e2e:
+        line["e2e"] = {"value": world * tokens_per_step * args.e2e_steps / e2e["seconds"], "unit": UNIT,
+                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": args.e2e_steps}
+    if world == 1 and not args.no_cpu_baseline:
+        cpu_prompt = make_prompt(cfg, 0, dev).to("cpu")
+        v, secs, desc = oracle_sample(cfg, cpu_prompt, keep, 1)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc,
+                                "cpu_seconds": secs}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

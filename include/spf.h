@@ -1,0 +1,159 @@
+/*
+ * spf.h -- C ABI of the speculative-prefill scoring / selection library for NVIDIA B200 (sm_100a).
+ *
+ * The library covers the data-parallel part of "Cross-Family Speculative Prefill" that runs between
+ * the draft model's forward pass and the assembly of the compressed prompt text:
+ *
+ *   spf_score          Appendix A.1.1 / Algorithm 1 "AggregateMaxMean": attention of the lookahead
+ *                      queries over the prompt keys, max over (layer, head), mean over lookahead.
+ *   spf_chunk_pool     Appendix A.1.2 / Algorithm 1 "AvgPool1D" + "PartitionIntoChunks": smoothing
+ *                      and per-chunk mean.
+ *   spf_select_topk    Appendix A.1.2 / Algorithm 1 "TopKChunks".
+ *   spf_compact_spans  Section 3.2 / Algorithm 1 "MergeAdjacentChunks" + "MapDraftChunksToTextSpans".
+ *
+ * Symbols: N prompt tokens (the paper's S), m lookahead queries (the paper's N), L layers, Hq query
+ * heads (the paper's H), Hkv key heads, G = Hq / Hkv, d head dimension, c chunk size, C = ceil(N / c),
+ * k chunks kept, w pooling kernel.
+ *
+ * General conventions
+ *   - Every pointer is DEVICE memory owned by the caller unless its comment says HOST.  The library
+ *     never frees or keeps caller memory and allocates nothing per call.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work is
+ *     enqueued on it; no call synchronises the stream or the device.
+ *   - Return value: SPF_OK (0) or a negative spf_status.  Argument checks happen on the host before
+ *     anything is launched; a failing call launches nothing.  spf_last_error() gives the text of the
+ *     calling thread's last failure.
+ *   - Conditions only the device can see are written to `dev_status` (see spf_score).
+ *   - Nothing here falls back to the CPU: unsupported shapes return SPF_ERR_UNSUPPORTED.
+ */
+#ifndef SPF_H_
+#define SPF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define SPF_API
+#else
+#define SPF_API __attribute__((visibility("default")))
+#endif
+
+typedef enum {
+  SPF_OK = 0,
+  SPF_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, misaligned K rows, k > C, ...      */
+  SPF_ERR_UNSUPPORTED = -2, /* shape outside what the kernels cover (see spf_score)                 */
+  SPF_ERR_WORKSPACE = -3,   /* workspace missing, misaligned or smaller than the size query says    */
+  SPF_ERR_CUDA = -4,        /* a CUDA runtime call failed (no device, launch error)                 */
+  SPF_ERR_TIMEOUT = -5      /* device status only: a bounded wait inside a kernel ran out           */
+} spf_status;
+
+/* Draft-model attention geometry shared by all prompts of a call. */
+typedef struct {
+  int32_t n_layers;     /* L >= 1                                                                  */
+  int32_t n_q_heads;    /* Hq, multiple of n_kv_heads                                              */
+  int32_t n_kv_heads;   /* Hkv                                                                     */
+  int32_t head_dim;     /* d: 64 or 128                                                            */
+  int32_t n_lookahead;  /* m: 1..32, with G * roundup(m, 8) <= 64                                   */
+  float softmax_scale;  /* multiplies q.k before the softmax; <= 0 selects 1/sqrt(d)                */
+} spf_shape;
+
+/* One prompt.  An array of these expresses a ragged batch; prompts are independent. */
+typedef struct {
+  int64_t n_tokens;            /* N >= 1                                                            */
+  const void* const* k_layers; /* HOST array of L device pointers; layer l is bf16 [Hkv][N][d],
+                                  post-RoPE, element (h, s, j) at h*k_stride_head + s*k_stride_tok + j */
+  int64_t k_stride_head;       /* in elements                                                       */
+  int64_t k_stride_tok;        /* in elements, >= d, multiple of 8 (rows start 16-byte aligned)     */
+  const void* q;               /* bf16 [L][Hq][m][d], contiguous, post-RoPE lookahead queries       */
+  float* importance;           /* out: fp32 [N], the token importance I                             */
+  float* lse;                  /* out, may be NULL: fp32 [L][Hq][m], natural-log sum-exp of each
+                                  softmax row, so that p = exp(scale * q.k - lse)                   */
+} spf_prompt;
+
+/*
+ * Bytes of scratch spf_score needs for these prompts (0 on invalid arguments; the reason is left in
+ * spf_last_error()).  The scratch holds packed queries, per-split softmax partials and row
+ * log-sum-exps; one buffer serves all prompts of the call in turn.
+ */
+SPF_API size_t spf_score_workspace_bytes(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts);
+
+/*
+ * Token importance (Appendix A.1.1; Algorithm 1, AggregateMaxMean).  For every prompt:
+ *     z[l,h,i,s] = scale * sum_j Q[l,h,i,j] * K[l, h / G, s, j]         (GQA: head h reads key head h / G)
+ *     p[l,h,i,s] = exp(z[l,h,i,s]) / sum_{s'} exp(z[l,h,i,s'])           softmax over the N prompt keys
+ *     A[i,s]     = max over all (l,h) of p[l,h,i,s]                      max over layer and head first,
+ *     I[s]       = (1/m) * sum_i A[i,s]                                  then the mean over lookahead
+ * written to prompts[p].importance (and the row log-sum-exps to prompts[p].lse when not NULL).
+ * bf16 inputs, fp32 accumulation and softmax.  The attention tensor itself is never stored.
+ *
+ * `shape`, `prompts` and the k_layers arrays are HOST memory, read during the call only.
+ * `workspace`: device, 256-byte aligned, at least spf_score_workspace_bytes(...) bytes; contents on
+ * entry are irrelevant, contents on exit unspecified.  Calls that share a workspace must be ordered
+ * on one stream.
+ * `dev_status`: device int32, may be NULL.  Kernels store a negative spf_status there when a
+ * device-side condition occurs (SPF_ERR_TIMEOUT from a bounded wait); they never trap.  The caller
+ * zeroes it before the call and reads it after synchronising.
+ * Errors: SPF_ERR_INVALID_ARG, SPF_ERR_UNSUPPORTED (d not 64/128, Hq % Hkv != 0, m > 32,
+ * G * roundup(m,8) > 64, L > 128), SPF_ERR_WORKSPACE, SPF_ERR_CUDA.
+ */
+SPF_API int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace,
+                          size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * Smoothing and chunk means (Appendix A.1.2; Algorithm 1, AvgPool1D and PartitionIntoChunks;
+ * kernel size 13 and chunk size 32 / 128 in Appendix A.3):
+ *     S[s]  = (1/w) * sum_{t = s - w/2}^{s + w/2} I[t]      terms outside [0, N) count as zero
+ *     cs[j] = mean of S over tokens [j*c, min((j+1)*c, N))
+ * importance: fp32 [N] in; chunk_scores: fp32 [ceil(N/c)] out.  pool_kernel w is odd, 1 <= w <= 255
+ * (1 = no smoothing); chunk c >= 1.
+ */
+SPF_API int32_t spf_chunk_pool(const float* importance, int64_t n_tokens, int32_t pool_kernel, int32_t chunk,
+                               float* chunk_scores, void* cuda_stream);
+
+/*
+ * Top-k chunks (Appendix A.1.2; Algorithm 1, TopKChunks): the indices of the k largest chunk scores,
+ * equal scores resolved toward the lower index, written in ascending order.
+ * chunk_scores: fp32 [n_chunks] in (finite); kept_chunks: int32 [k] out; 1 <= k <= n_chunks < 2^31.
+ */
+SPF_API int32_t spf_select_topk(const float* chunk_scores, int64_t n_chunks, int64_t k, int32_t* kept_chunks,
+                                void* cuda_stream);
+
+/*
+ * Merge and compaction (Section 3.2; Algorithm 1, MergeAdjacentChunks and MapDraftChunksToTextSpans).
+ * kept_chunks: int32 [k], ascending, distinct, each in [0, ceil(N/c)) -- as spf_select_topk writes them.
+ * Runs of consecutive kept chunks become one token span [a, b) (b clipped to N); its character span
+ * is [char_start[a], char_end[b-1]).  Kept tokens keep their original order.
+ *   token_ids, char_start, char_end : int32 [N] in (character offsets of each draft token in the text)
+ *   out_ids        int32 [>= min(k*c, N)]  kept token ids, n_kept of them
+ *   out_pos        int32 [>= min(k*c, N)]  their original positions; may be NULL
+ *   out_tok_spans  int32 [k][2]            n_spans rows (a, b)
+ *   out_char_spans int32 [k][2]            n_spans rows (char_start[a], char_end[b-1])
+ *   out_counts     int64 [2]               {n_kept, n_spans}
+ * Rows beyond n_kept / n_spans are left untouched.
+ */
+SPF_API int32_t spf_compact_spans(const int32_t* kept_chunks, int64_t k, int32_t chunk, int64_t n_tokens,
+                                  const int32_t* token_ids, const int32_t* char_start, const int32_t* char_end,
+                                  int32_t* out_ids, int32_t* out_pos, int32_t* out_tok_spans,
+                                  int32_t* out_char_spans, int64_t* out_counts, void* cuda_stream);
+
+/*
+ * Host helper for the keep rate of Section 3.1: the number of chunks a keep rate rho retains,
+ * clamp(ceil(rho * n_chunks), 1, n_chunks).  Pure host arithmetic; returns 0 if n_chunks < 1.
+ */
+SPF_API int64_t spf_keep_count(int64_t n_chunks, double keep_ratio);
+
+/* Text of a status code (static storage). */
+SPF_API const char* spf_status_string(int32_t status);
+/* Text of the calling thread's most recent failure ("" if none).  Thread-local storage. */
+SPF_API const char* spf_last_error(void);
+/* Library version, e.g. "0.1.0". */
+SPF_API const char* spf_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPF_H_ */

@@ -1,0 +1,297 @@
+"""ctypes binding of ``include/spf.h``: argument marshalling only.
+
+The functions named ``spf_*`` mirror the C entry points one to one and take torch CUDA tensors
+(used here as device buffers) instead of raw pointers.  ``Selector`` chains the four calls for one
+prompt and owns the scratch buffers a serving loop would reuse.
+"""
+from __future__ import annotations
+
+import ctypes
+import dataclasses
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(PKG_DIR, "libspf.so")
+
+
+class SpfError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str):
+        super().__init__(f"{where}: status {status} ({detail})")
+        self.status = status
+
+
+class _Shape(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("n_lookahead", ctypes.c_int32), ("softmax_scale", ctypes.c_float)]
+
+
+class _Prompt(ctypes.Structure):
+    _fields_ = [("n_tokens", ctypes.c_int64), ("k_layers", ctypes.POINTER(ctypes.c_void_p)),
+                ("k_stride_head", ctypes.c_int64), ("k_stride_tok", ctypes.c_int64), ("q", ctypes.c_void_p),
+                ("importance", ctypes.c_void_p), ("lse", ctypes.c_void_p)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2603_02631_b200.build` "
+                          "(there is no fallback path)")
+    dll = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    dll.spf_score_workspace_bytes.restype = ctypes.c_size_t
+    dll.spf_score_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32]
+    dll.spf_score.restype = i32
+    dll.spf_score.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp, ctypes.c_size_t, vp, vp]
+    dll.spf_chunk_pool.restype = i32
+    dll.spf_chunk_pool.argtypes = [vp, i64, i32, i32, vp, vp]
+    dll.spf_select_topk.restype = i32
+    dll.spf_select_topk.argtypes = [vp, i64, i64, vp, vp]
+    dll.spf_compact_spans.restype = i32
+    dll.spf_compact_spans.argtypes = [vp, i64, i32, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    dll.spf_keep_count.restype = i64
+    dll.spf_keep_count.argtypes = [i64, ctypes.c_double]
+    dll.spf_status_string.restype = ctypes.c_char_p
+    dll.spf_status_string.argtypes = [i32]
+    dll.spf_last_error.restype = ctypes.c_char_p
+    dll.spf_last_error.argtypes = []
+    dll.spf_version.restype = ctypes.c_char_p
+    dll.spf_version.argtypes = []
+    return dll
+
+
+lib = _load()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise SpfError(status, where, (lib.spf_last_error() or b"").decode() or
+                       (lib.spf_status_string(status) or b"").decode())
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype:
+        raise TypeError(f"{name} must be a CUDA tensor of dtype {dtype}")
+    return t
+
+
+def spf_version() -> str:
+    return lib.spf_version().decode()
+
+
+def spf_status_string(status: int) -> str:
+    return lib.spf_status_string(status).decode()
+
+
+def spf_last_error() -> str:
+    return lib.spf_last_error().decode()
+
+
+def spf_keep_count(n_chunks: int, keep_ratio: float) -> int:
+    return int(lib.spf_keep_count(n_chunks, keep_ratio))
+
+
+@dataclasses.dataclass
+class PromptBuffers:
+    """Device buffers of one prompt, as spf_score reads and writes them."""
+    q: torch.Tensor                      # bf16 [L, Hq, m, d]
+    k_layers: Sequence[torch.Tensor]     # L tensors bf16 [Hkv, N, d]; last dim contiguous
+    importance: torch.Tensor             # fp32 [N] (out)
+    lse: Optional[torch.Tensor] = None   # fp32 [L, Hq, m] (out)
+
+
+def _marshal(prompts: Sequence[PromptBuffers], softmax_scale: float):
+    first = prompts[0]
+    L, Hq, m, d = first.q.shape
+    Hkv = first.k_layers[0].shape[0]
+    shape = _Shape(L, Hq, Hkv, d, m, float(softmax_scale))
+    arr = (_Prompt * len(prompts))()
+    keep = []
+    for i, p in enumerate(prompts):
+        _dev(p.q, torch.bfloat16, "q")
+        if tuple(p.q.shape) != (L, Hq, m, d) or not p.q.is_contiguous():
+            raise ValueError("q must be contiguous [L, Hq, m, d], the same shape for all prompts")
+        if len(p.k_layers) != L:
+            raise ValueError("k_layers must hold one tensor per layer")
+        k0 = p.k_layers[0]
+        n = k0.shape[1]
+        for kl in p.k_layers:
+            _dev(kl, torch.bfloat16, "k_layers[l]")
+            if tuple(kl.shape) != (Hkv, n, d) or kl.stride(2) != 1 or kl.stride() != k0.stride():
+                raise ValueError("every k_layers[l] must be [Hkv, N, d] with a contiguous last dim and equal strides")
+        _dev(p.importance, torch.float32, "importance")
+        if p.importance.numel() != n or not p.importance.is_contiguous():
+            raise ValueError("importance must be contiguous fp32 [N]")
+        if p.lse is not None:
+            _dev(p.lse, torch.float32, "lse")
+            if p.lse.numel() != L * Hq * m or not p.lse.is_contiguous():
+                raise ValueError("lse must be contiguous fp32 [L, Hq, m]")
+        ptrs = (ctypes.c_void_p * L)(*[kl.data_ptr() for kl in p.k_layers])
+        keep.append(ptrs)
+        arr[i] = _Prompt(n, ctypes.cast(ptrs, ctypes.POINTER(ctypes.c_void_p)), k0.stride(0), k0.stride(1),
+                         p.q.data_ptr(), p.importance.data_ptr(), _ptr(p.lse))
+    return shape, arr, keep
+
+
+def spf_score_workspace_bytes(prompts: Sequence[PromptBuffers], softmax_scale: float = 0.0) -> int:
+    shape, arr, _keep = _marshal(prompts, softmax_scale)
+    n = int(lib.spf_score_workspace_bytes(ctypes.byref(shape), arr, len(prompts)))
+    if n == 0:
+        raise SpfError(-1, "spf_score_workspace_bytes", spf_last_error())
+    return n
+
+
+def spf_score(prompts: Sequence[PromptBuffers], workspace: torch.Tensor, softmax_scale: float = 0.0,
+              dev_status: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> None:
+    shape, arr, _keep = _marshal(prompts, softmax_scale)
+    if not workspace.is_cuda:
+        raise TypeError("workspace must be a CUDA tensor")
+    _check(lib.spf_score(ctypes.byref(shape), arr, len(prompts), workspace.data_ptr(),
+                         workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
+           "spf_score")
+
+
+def spf_chunk_pool(importance: torch.Tensor, pool_kernel: int, chunk: int, chunk_scores: torch.Tensor,
+                   stream: Optional[torch.cuda.Stream] = None) -> None:
+    _dev(importance, torch.float32, "importance")
+    _dev(chunk_scores, torch.float32, "chunk_scores")
+    n = importance.numel()
+    if chunk >= 1 and chunk_scores.numel() < (n + chunk - 1) // chunk:
+        raise ValueError("chunk_scores is too small")
+    _check(lib.spf_chunk_pool(importance.data_ptr(), n, pool_kernel, chunk, chunk_scores.data_ptr(),
+                              _stream_ptr(stream)), "spf_chunk_pool")
+
+
+def spf_select_topk(chunk_scores: torch.Tensor, n_chunks: int, k: int, kept_chunks: torch.Tensor,
+                    stream: Optional[torch.cuda.Stream] = None) -> None:
+    _dev(chunk_scores, torch.float32, "chunk_scores")
+    _dev(kept_chunks, torch.int32, "kept_chunks")
+    if chunk_scores.numel() < n_chunks or kept_chunks.numel() < k:
+        raise ValueError("chunk_scores or kept_chunks is too small")
+    _check(lib.spf_select_topk(chunk_scores.data_ptr(), n_chunks, k, kept_chunks.data_ptr(), _stream_ptr(stream)),
+           "spf_select_topk")
+
+
+def spf_compact_spans(kept_chunks: torch.Tensor, k: int, chunk: int, n_tokens: int, token_ids: torch.Tensor,
+                      char_start: torch.Tensor, char_end: torch.Tensor, out_ids: torch.Tensor,
+                      out_pos: Optional[torch.Tensor], out_tok_spans: torch.Tensor, out_char_spans: torch.Tensor,
+                      out_counts: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    for name, t in (("kept_chunks", kept_chunks), ("token_ids", token_ids), ("char_start", char_start),
+                    ("char_end", char_end), ("out_ids", out_ids), ("out_tok_spans", out_tok_spans),
+                    ("out_char_spans", out_char_spans)):
+        _dev(t, torch.int32, name)
+    if out_pos is not None:
+        _dev(out_pos, torch.int32, "out_pos")
+    _dev(out_counts, torch.int64, "out_counts")
+    need = min(max(k, 0) * max(chunk, 0), n_tokens)
+    if out_ids.numel() < need or (out_pos is not None and out_pos.numel() < need) or \
+            out_tok_spans.numel() < 2 * k or out_char_spans.numel() < 2 * k or out_counts.numel() < 2 or \
+            min(token_ids.numel(), char_start.numel(), char_end.numel()) < n_tokens or kept_chunks.numel() < k:
+        raise ValueError("a buffer is smaller than include/spf.h requires")
+    _check(lib.spf_compact_spans(kept_chunks.data_ptr(), k, chunk, n_tokens, token_ids.data_ptr(),
+                                 char_start.data_ptr(), char_end.data_ptr(), out_ids.data_ptr(), _ptr(out_pos),
+                                 out_tok_spans.data_ptr(), out_char_spans.data_ptr(), out_counts.data_ptr(),
+                                 _stream_ptr(stream)), "spf_compact_spans")
+
+
+@dataclasses.dataclass
+class Selection:
+    """Device-side result of one prompt; ``n_kept`` / ``n_spans`` are read from ``counts`` on demand."""
+    importance: torch.Tensor
+    lse: torch.Tensor
+    chunk_scores: torch.Tensor
+    k: int
+    kept_chunks: torch.Tensor
+    out_ids: torch.Tensor
+    out_pos: torch.Tensor
+    tok_spans: torch.Tensor
+    char_spans: torch.Tensor
+    counts: torch.Tensor
+
+    def host(self):
+        """Copies the result to the host (synchronises) and trims it to the valid rows."""
+        counts = self.counts.cpu()
+        n_kept, n_spans = int(counts[0]), int(counts[1])
+        return dict(importance=self.importance.cpu().numpy(), lse=self.lse.cpu().numpy(),
+                    chunk_scores=self.chunk_scores.cpu().numpy(), k=self.k,
+                    kept=self.kept_chunks[:self.k].cpu().numpy(), ids=self.out_ids[:n_kept].cpu().numpy(),
+                    pos=self.out_pos[:n_kept].cpu().numpy(), tok_spans=self.tok_spans[:n_spans].cpu().numpy(),
+                    char_spans=self.char_spans[:n_spans].cpu().numpy())
+
+
+class Selector:
+    """Chains spf_score -> spf_chunk_pool -> spf_select_topk -> spf_compact_spans for prompts of one geometry.
+
+    Buffers are allocated once for ``max_tokens`` and reused, so that a call enqueues kernels only.
+    """
+
+    def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n_lookahead: int,
+                 max_tokens: int, chunk: int = 32, pool_kernel: int = 13, softmax_scale: float = 0.0,
+                 device: str = "cuda"):
+        self.geom = (n_layers, n_q_heads, n_kv_heads, head_dim, n_lookahead)
+        self.chunk, self.pool_kernel, self.softmax_scale = chunk, pool_kernel, softmax_scale
+        self.max_tokens = max_tokens
+        self.device = torch.device(device)
+        max_chunks = (max_tokens + chunk - 1) // chunk
+        dev = self.device
+        self.importance = torch.empty(max_tokens, dtype=torch.float32, device=dev)
+        self.lse = torch.empty(n_layers * n_q_heads * n_lookahead, dtype=torch.float32, device=dev)
+        self.chunk_scores = torch.empty(max_chunks, dtype=torch.float32, device=dev)
+        self.kept = torch.empty(max_chunks, dtype=torch.int32, device=dev)
+        self.out_ids = torch.empty(max_tokens, dtype=torch.int32, device=dev)
+        self.out_pos = torch.empty(max_tokens, dtype=torch.int32, device=dev)
+        self.tok_spans = torch.empty((max_chunks, 2), dtype=torch.int32, device=dev)
+        self.char_spans = torch.empty((max_chunks, 2), dtype=torch.int32, device=dev)
+        self.counts = torch.zeros(2, dtype=torch.int64, device=dev)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.workspace: Optional[torch.Tensor] = None
+
+    def _workspace(self, bufs: PromptBuffers) -> torch.Tensor:
+        need = spf_score_workspace_bytes([bufs], self.softmax_scale)
+        if self.workspace is None or self.workspace.numel() < need:
+            self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        return self.workspace
+
+    def run(self, q: torch.Tensor, k_layers: Sequence[torch.Tensor], token_ids: torch.Tensor,
+            char_start: torch.Tensor, char_end: torch.Tensor, keep: float,
+            stream: Optional[torch.cuda.Stream] = None) -> Selection:
+        """Enqueues the whole path for one prompt whose tensors are already on the device."""
+        n = k_layers[0].shape[1]
+        if n > self.max_tokens:
+            raise ValueError(f"prompt has {n} tokens, selector was sized for {self.max_tokens}")
+        n_chunks = (n + self.chunk - 1) // self.chunk
+        k = spf_keep_count(n_chunks, keep)
+        bufs = PromptBuffers(q, k_layers, self.importance[:n], self.lse)
+        spf_score([bufs], self._workspace(bufs), self.softmax_scale, self.dev_status, stream)
+        spf_chunk_pool(self.importance[:n], self.pool_kernel, self.chunk, self.chunk_scores[:n_chunks], stream)
+        spf_select_topk(self.chunk_scores, n_chunks, k, self.kept, stream)
+        spf_compact_spans(self.kept, k, self.chunk, n, token_ids, char_start, char_end, self.out_ids, self.out_pos,
+                          self.tok_spans, self.char_spans, self.counts, stream)
+        L, Hq, _, _, m = self.geom
+        return Selection(self.importance[:n], self.lse.view(L, Hq, m), self.chunk_scores[:n_chunks], k, self.kept,
+                         self.out_ids, self.out_pos, self.tok_spans, self.char_spans, self.counts)
+
+    def run_host(self, q: torch.Tensor, k_layers: Sequence[torch.Tensor], token_ids: torch.Tensor,
+                 char_start: torch.Tensor, char_end: torch.Tensor, keep: float):
+        """Same path for HOST tensors (ideally pinned): copies in, runs, copies the selection back.
+
+        Returns host NumPy arrays: kept ids, positions, token spans, character spans.
+        """
+        dev = self.device
+        qd = q.to(dev, non_blocking=True)
+        kd = [t.to(dev, non_blocking=True) for t in k_layers]
+        idd, csd, ced = (t.to(dev, non_blocking=True) for t in (token_ids, char_start, char_end))
+        sel = self.run(qd, kd, idd, csd, ced, keep)
+        counts = sel.counts.cpu()
+        n_kept, n_spans = int(counts[0]), int(counts[1])
+        return dict(ids=sel.out_ids[:n_kept].cpu().numpy(), pos=sel.out_pos[:n_kept].cpu().numpy(),
+                    tok_spans=sel.tok_spans[:n_spans].cpu().numpy(), char_spans=sel.char_spans[:n_spans].cpu().numpy())

@@ -1,0 +1,167 @@
+// Host side of the C ABI: argument validation, error text, dispatch of spf_score.
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+#include "score.cuh"
+
+namespace spf {
+namespace {
+
+thread_local char g_error[512] = "";
+
+// Builds the per-prompt problem description; returns a status and leaves the reason in the error text.
+int32_t make_problem(const spf_shape* shape, const spf_prompt& pr, int32_t index, ScoreProblem* out) {
+  ScoreProblem p{};
+  p.n_layers = shape->n_layers;
+  p.n_q_heads = shape->n_q_heads;
+  p.n_kv_heads = shape->n_kv_heads;
+  p.head_dim = shape->head_dim;
+  p.n_lookahead = shape->n_lookahead;
+  if (p.n_layers < 1 || p.n_q_heads < 1 || p.n_kv_heads < 1 || p.n_lookahead < 1)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score: shape fields must be positive");
+  if (p.n_layers > kMaxLayers) return fail(SPF_ERR_UNSUPPORTED, "spf_score: n_layers %d > %d", p.n_layers, kMaxLayers);
+  if (p.head_dim != 64 && p.head_dim != 128)
+    return fail(SPF_ERR_UNSUPPORTED, "spf_score: head_dim must be 64 or 128 (got %d)", p.head_dim);
+  if (p.n_q_heads % p.n_kv_heads != 0)
+    return fail(SPF_ERR_UNSUPPORTED, "spf_score: n_q_heads %d is not a multiple of n_kv_heads %d", p.n_q_heads, p.n_kv_heads);
+  p.group = p.n_q_heads / p.n_kv_heads;
+  if (p.n_lookahead > 32) return fail(SPF_ERR_UNSUPPORTED, "spf_score: n_lookahead %d > 32", p.n_lookahead);
+  p.m_pad = (p.n_lookahead + 7) / 8 * 8;
+  if (p.group * p.m_pad > 64)
+    return fail(SPF_ERR_UNSUPPORTED, "spf_score: group %d x lookahead %d (padded to %d) exceeds 64 query rows per kv head",
+                p.group, p.n_lookahead, p.m_pad);
+  p.rows_pad = (p.group * p.m_pad + 15) / 16 * 16;
+  const float scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.0f / std::sqrt((float)p.head_dim);
+  if (!std::isfinite(scale)) return fail(SPF_ERR_INVALID_ARG, "spf_score: softmax_scale is not finite");
+  p.c_log2 = scale * kLog2e;
+
+  if (pr.n_tokens < 1) return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: n_tokens must be >= 1", index);
+  if (pr.n_tokens > 0x7fffffffLL) return fail(SPF_ERR_UNSUPPORTED, "spf_score: prompt %d: n_tokens >= 2^31", index);
+  if (pr.k_layers == nullptr || pr.q == nullptr || pr.importance == nullptr)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: null pointer", index);
+  if (pr.k_stride_tok < p.head_dim || pr.k_stride_tok % 8 != 0)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: k_stride_tok %lld must be >= head_dim and a multiple of 8", index,
+                (long long)pr.k_stride_tok);
+  if (pr.k_stride_head % 8 != 0 || (p.n_kv_heads > 1 && pr.k_stride_head < 1))
+    return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: k_stride_head %lld must be positive and a multiple of 8", index,
+                (long long)pr.k_stride_head);
+  if (reinterpret_cast<uintptr_t>(pr.q) % 4 != 0)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: q is not 4-byte aligned", index);
+  for (int l = 0; l < p.n_layers; ++l) {
+    const void* kp = pr.k_layers[l];
+    if (kp == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: k_layers[%d] is null", index, l);
+    if (reinterpret_cast<uintptr_t>(kp) % 16 != 0)
+      return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: k_layers[%d] is not 16-byte aligned", index, l);
+    p.k.p[l] = static_cast<const __nv_bfloat16*>(kp);
+  }
+  p.n_tokens = pr.n_tokens;
+  p.stride_head = pr.k_stride_head;
+  p.stride_tok = pr.k_stride_tok;
+  p.q = static_cast<const __nv_bfloat16*>(pr.q);
+  p.importance = pr.importance;
+  p.lse_out = pr.lse;
+  *out = p;
+  return SPF_OK;
+}
+
+int32_t device_sm_count(int* out) {
+  int dev = 0;
+  SPF_CUDA_CHECK(cudaGetDevice(&dev));
+  static std::mutex mu;
+  static int cached[64];
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev < 0 || dev >= 64) return fail(SPF_ERR_CUDA, "device ordinal %d out of range", dev);
+  if (cached[dev] == 0) SPF_CUDA_CHECK(cudaDeviceGetAttribute(&cached[dev], cudaDevAttrMultiProcessorCount, dev));
+  *out = cached[dev];
+  return SPF_OK;
+}
+
+}  // namespace
+
+int32_t fail(int32_t code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_error, sizeof(g_error), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+void clear_error() { g_error[0] = '\0'; }
+
+}  // namespace spf
+
+using namespace spf;
+
+extern "C" size_t spf_score_workspace_bytes(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts) {
+  clear_error();
+  if (shape == nullptr || prompts == nullptr || n_prompts < 1) {
+    fail(SPF_ERR_INVALID_ARG, "spf_score_workspace_bytes: null argument or n_prompts < 1");
+    return 0;
+  }
+  size_t need = 0;
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    if (make_problem(shape, prompts[i], i, &p) != SPF_OK) return 0;
+    need = std::max(need, score_mma_workspace_bytes(p));
+  }
+  return need;
+}
+
+extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace,
+                             size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  clear_error();
+  (void)dev_status;  // the two-sweep path has no device-side wait that could run out
+  if (shape == nullptr || prompts == nullptr || n_prompts < 1)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score: null argument or n_prompts < 1");
+  // validate everything before the first launch
+  size_t need = 0;
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    const int32_t st = make_problem(shape, prompts[i], i, &p);
+    if (st != SPF_OK) return st;
+    need = std::max(need, score_mma_workspace_bytes(p));
+  }
+  if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
+    return fail(SPF_ERR_WORKSPACE, "spf_score: workspace is null or not 256-byte aligned");
+  if (workspace_bytes < need)
+    return fail(SPF_ERR_WORKSPACE, "spf_score: workspace has %zu bytes, %zu needed", workspace_bytes, need);
+  int sm_count = 0;
+  {
+    const int32_t st = device_sm_count(&sm_count);
+    if (st != SPF_OK) return st;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    make_problem(shape, prompts[i], i, &p);
+    const int32_t st = score_mma_launch(p, workspace, sm_count, stream);
+    if (st != SPF_OK) return st;
+  }
+  return SPF_OK;
+}
+
+extern "C" int64_t spf_keep_count(int64_t n_chunks, double keep_ratio) {
+  if (n_chunks < 1) return 0;
+  if (!(keep_ratio > 0.0)) return 1;
+  const double want = std::ceil(keep_ratio * (double)n_chunks - 1e-9);
+  if (want >= (double)n_chunks) return n_chunks;
+  return want < 1.0 ? 1 : (int64_t)want;
+}
+
+extern "C" const char* spf_status_string(int32_t status) {
+  switch (status) {
+    case SPF_OK: return "ok";
+    case SPF_ERR_INVALID_ARG: return "invalid argument";
+    case SPF_ERR_UNSUPPORTED: return "unsupported shape";
+    case SPF_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case SPF_ERR_CUDA: return "CUDA runtime error";
+    case SPF_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+extern "C" const char* spf_last_error(void) { return g_error; }
+
+extern "C" const char* spf_version(void) { return "0.1.0"; }

@@ -1,0 +1,26 @@
+// Internal description of one prompt's scoring problem and the entry points of the scoring paths.
+#pragma once
+
+#include "common.cuh"
+
+namespace spf {
+
+struct ScoreProblem {
+  int n_layers, n_q_heads, n_kv_heads, group, head_dim, n_lookahead;
+  int m_pad;     // n_lookahead rounded up to a multiple of 8
+  int rows_pad;  // group * m_pad rounded up to a multiple of 16: query rows per kv-head tile
+  float c_log2;  // softmax scale times log2(e): logits are handled in base-2 units
+  int64_t n_tokens, stride_head, stride_tok;
+  LayerPtrs k;
+  const __nv_bfloat16* q;
+  float* importance;
+  float* lse_out;  // may be null
+};
+
+constexpr int kMmaMaxSplit = 64;  // upper bound on the key splits of sweep 1 (sizes the partials buffer)
+
+// General two-sweep path (warp-level mma.sync tiles, key cache read twice).
+size_t score_mma_workspace_bytes(const ScoreProblem& p);
+int32_t score_mma_launch(const ScoreProblem& p, void* workspace, int sm_count, cudaStream_t stream);
+
+}  // namespace spf

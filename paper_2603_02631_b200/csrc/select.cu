@@ -1,0 +1,248 @@
+// Chunk pooling, top-k chunk selection and span compaction (Appendix A.1.2, Section 3.2).
+// These steps touch a few hundred KB at most; they are latency-bound and each is a single launch.
+#include "common.cuh"
+
+namespace spf {
+namespace {
+
+// ------------------------------------------------------------------------------------------------
+// spf_chunk_pool: one warp per chunk.  Each lane sums the w-wide windows of its tokens, the warp adds
+// them up in a fixed order, so the result does not depend on scheduling.
+// ------------------------------------------------------------------------------------------------
+constexpr int kPoolWarps = 8;
+
+__global__ void __launch_bounds__(kPoolWarps * 32) chunk_pool_kernel(const float* __restrict__ importance, int64_t n_tokens,
+                                                                      int half, float inv_w, int chunk,
+                                                                      float* __restrict__ chunk_scores, int64_t n_chunks) {
+  const int lane = threadIdx.x & 31;
+  const int64_t j = (int64_t)blockIdx.x * kPoolWarps + (threadIdx.x >> 5);
+  if (j >= n_chunks) return;
+  const int64_t lo = j * chunk;
+  const int64_t hi = min(lo + (int64_t)chunk, n_tokens);
+  float sum = 0.f;
+  for (int64_t s = lo + lane; s < hi; s += 32) {
+    const int64_t a = max(s - half, (int64_t)0), b = min(s + half, n_tokens - 1);
+    float win = 0.f;
+    for (int64_t t = a; t <= b; ++t) win += __ldg(importance + t);
+    sum += win * inv_w;
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+  if (lane == 0) chunk_scores[j] = sum / (float)(hi - lo);
+}
+
+// ------------------------------------------------------------------------------------------------
+// spf_select_topk: one CTA.  Scores map to unsigned keys whose integer order is the float order; a
+// four-pass radix select (8 bits per pass, most significant first) finds the k-th largest key; then
+// everything above it, plus the lowest-index entries equal to it, is written out in index order.
+// ------------------------------------------------------------------------------------------------
+constexpr int kTopkThreads = 1024;
+
+__device__ __forceinline__ uint32_t order_key(float x) {
+  x += 0.0f;  // -0 -> +0 so that the two zeros tie
+  const uint32_t b = __float_as_uint(x);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Exclusive prefix count of `flag` over the CTA (thread order); *total gets the CTA-wide count.
+__device__ __forceinline__ int block_exclusive_count(bool flag, int* warp_counts, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned ballot = __ballot_sync(0xffffffffu, flag);
+  const int within = __popc(ballot & ((1u << lane) - 1u));
+  __syncthreads();  // warp_counts may still be read from the previous use
+  if (lane == 0) warp_counts[warp] = __popc(ballot);
+  __syncthreads();
+  int before = 0, all = 0;
+  for (int w = 0; w < kTopkThreads / 32; ++w) {
+    const int cnt = warp_counts[w];
+    before += w < warp ? cnt : 0;
+    all += cnt;
+  }
+  *total = all;
+  return before + within;
+}
+
+__global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* __restrict__ scores, int n, int k,
+                                                                    int32_t* __restrict__ kept) {
+  __shared__ int hist[256];
+  __shared__ int warp_counts[kTopkThreads / 32];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_remaining;
+
+  uint32_t prefix = 0;     // the bits of the k-th largest key found so far
+  uint32_t mask = 0;       // which bits of `prefix` are fixed
+  int remaining = k;       // rank of the wanted key among the keys that match the prefix
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int b = threadIdx.x; b < 256; b += kTopkThreads) hist[b] = 0;
+    __syncthreads();
+    for (int j = threadIdx.x; j < n; j += kTopkThreads) {
+      const uint32_t key = order_key(scores[j]);
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int rem = remaining, b = 255;
+      for (; b > 0; --b) {
+        if (hist[b] >= rem) break;
+        rem -= hist[b];
+      }
+      sh_prefix = prefix | ((uint32_t)b << shift);
+      sh_remaining = rem;
+    }
+    __syncthreads();
+    prefix = sh_prefix;
+    remaining = sh_remaining;
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  // `prefix` is now the k-th largest key; `remaining` of the entries equal to it are kept (lowest indices).
+  int out_base = 0, eq_base = 0;
+  for (int j0 = 0; j0 < n; j0 += kTopkThreads) {
+    const int j = j0 + threadIdx.x;
+    const uint32_t key = j < n ? order_key(scores[j]) : 0u;
+    const bool gt = j < n && key > prefix;
+    const bool eq = j < n && key == prefix;
+    int eq_total, sel_total;
+    const int eq_rank = eq_base + block_exclusive_count(eq, warp_counts, &eq_total);
+    const bool sel = gt || (eq && eq_rank < remaining);
+    const int pos = out_base + block_exclusive_count(sel, warp_counts, &sel_total);
+    if (sel && pos < k) kept[pos] = j;
+    out_base += sel_total;
+    eq_base += eq_total;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// spf_compact_spans.  Kept chunk r (ascending order) starts at output offset r * c because only the
+// very last chunk of the prompt can be short and, if kept, it is the last one kept.  Block 0 finds
+// the runs of consecutive chunks (a prefix count of run starts) and writes the spans and counts; the
+// other blocks copy ids and positions, one warp per kept chunk.
+// ------------------------------------------------------------------------------------------------
+constexpr int kCompactThreads = 256;
+
+__global__ void __launch_bounds__(kCompactThreads) compact_spans_kernel(
+    const int32_t* __restrict__ kept, int k, int chunk, int64_t n_tokens, const int32_t* __restrict__ token_ids,
+    const int32_t* __restrict__ char_start, const int32_t* __restrict__ char_end, int32_t* __restrict__ out_ids,
+    int32_t* __restrict__ out_pos, int32_t* __restrict__ out_tok_spans, int32_t* __restrict__ out_char_spans,
+    int64_t* __restrict__ out_counts) {
+  const int64_t n_chunks = (n_tokens + chunk - 1) / chunk;
+  if (blockIdx.x == 0) {
+    __shared__ int warp_counts[kCompactThreads / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int span_base = 0;
+    for (int r0 = 0; r0 < k; r0 += kCompactThreads) {
+      const int r = r0 + threadIdx.x;
+      int64_t j = -1;
+      bool starts = false, ends = false;
+      if (r < k) {
+        j = kept[r];
+        starts = r == 0 || kept[r - 1] + 1 != j;
+        ends = r == k - 1 || kept[r + 1] != j + 1;
+      }
+      const unsigned ballot = __ballot_sync(0xffffffffu, starts);
+      const int within = __popc(ballot & ((2u << lane) - 1u));  // inclusive
+      __syncthreads();
+      if (lane == 0) warp_counts[warp] = __popc(ballot);
+      __syncthreads();
+      int before = 0, all = 0;
+      for (int w = 0; w < kCompactThreads / 32; ++w) {
+        before += w < warp ? warp_counts[w] : 0;
+        all += warp_counts[w];
+      }
+      const int span = span_base + before + within - 1;  // index of the run this chunk belongs to
+      if (r < k && j >= 0 && j < n_chunks) {
+        if (starts) {
+          const int64_t a = j * chunk;
+          out_tok_spans[2 * span] = (int32_t)a;
+          out_char_spans[2 * span] = char_start[a];
+        }
+        if (ends) {
+          const int64_t b = min((j + 1) * chunk, n_tokens);
+          out_tok_spans[2 * span + 1] = (int32_t)b;
+          out_char_spans[2 * span + 1] = char_end[b - 1];
+        }
+      }
+      span_base += all;
+    }
+    if (threadIdx.x == 0) {
+      const int64_t last = kept[k - 1];
+      const int64_t last_size = min((last + 1) * chunk, n_tokens) - last * chunk;
+      out_counts[0] = (int64_t)(k - 1) * chunk + last_size;
+      out_counts[1] = span_base;
+    }
+    return;
+  }
+  const int warps = kCompactThreads / 32;
+  const int lane = threadIdx.x & 31;
+  const int64_t r = (int64_t)(blockIdx.x - 1) * warps + (threadIdx.x >> 5);
+  if (r >= k) return;
+  const int64_t j = kept[r];
+  if (j < 0 || j >= n_chunks) return;
+  const int64_t lo = j * chunk, hi = min(lo + chunk, n_tokens);
+  for (int64_t s = lo + lane; s < hi; s += 32) {
+    const int64_t o = r * chunk + (s - lo);
+    out_ids[o] = token_ids[s];
+    if (out_pos != nullptr) out_pos[o] = (int32_t)s;
+  }
+}
+
+}  // namespace
+}  // namespace spf
+
+using namespace spf;
+
+extern "C" int32_t spf_chunk_pool(const float* importance, int64_t n_tokens, int32_t pool_kernel, int32_t chunk,
+                                  float* chunk_scores, void* cuda_stream) {
+  clear_error();
+  if (importance == nullptr || chunk_scores == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool: null pointer");
+  if (n_tokens < 1) return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool: n_tokens must be >= 1 (got %lld)", (long long)n_tokens);
+  if (pool_kernel < 1 || pool_kernel > 255 || pool_kernel % 2 == 0)
+    return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool: pool_kernel must be odd and in [1, 255] (got %d)", pool_kernel);
+  if (chunk < 1) return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool: chunk must be >= 1 (got %d)", chunk);
+  const int64_t n_chunks = ceil_div(n_tokens, chunk);
+  const int64_t blocks = ceil_div(n_chunks, kPoolWarps);
+  if (blocks > 0x7fffffff) return fail(SPF_ERR_UNSUPPORTED, "spf_chunk_pool: too many chunks");
+  chunk_pool_kernel<<<(unsigned)blocks, kPoolWarps * 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      importance, n_tokens, pool_kernel / 2, 1.0f / (float)pool_kernel, chunk, chunk_scores, n_chunks);
+  SPF_CUDA_CHECK(cudaGetLastError());
+  return SPF_OK;
+}
+
+extern "C" int32_t spf_select_topk(const float* chunk_scores, int64_t n_chunks, int64_t k, int32_t* kept_chunks,
+                                   void* cuda_stream) {
+  clear_error();
+  if (chunk_scores == nullptr || kept_chunks == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_select_topk: null pointer");
+  if (n_chunks < 1 || n_chunks > 0x7fffffff)
+    return fail(SPF_ERR_INVALID_ARG, "spf_select_topk: n_chunks must be in [1, 2^31) (got %lld)", (long long)n_chunks);
+  if (k < 1 || k > n_chunks)
+    return fail(SPF_ERR_INVALID_ARG, "spf_select_topk: k must be in [1, n_chunks] (got k=%lld, n_chunks=%lld)", (long long)k,
+                (long long)n_chunks);
+  select_topk_kernel<<<1, kTopkThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(chunk_scores, (int)n_chunks, (int)k,
+                                                                                    kept_chunks);
+  SPF_CUDA_CHECK(cudaGetLastError());
+  return SPF_OK;
+}
+
+extern "C" int32_t spf_compact_spans(const int32_t* kept_chunks, int64_t k, int32_t chunk, int64_t n_tokens,
+                                     const int32_t* token_ids, const int32_t* char_start, const int32_t* char_end,
+                                     int32_t* out_ids, int32_t* out_pos, int32_t* out_tok_spans, int32_t* out_char_spans,
+                                     int64_t* out_counts, void* cuda_stream) {
+  clear_error();
+  if (kept_chunks == nullptr || token_ids == nullptr || char_start == nullptr || char_end == nullptr || out_ids == nullptr ||
+      out_tok_spans == nullptr || out_char_spans == nullptr || out_counts == nullptr)
+    return fail(SPF_ERR_INVALID_ARG, "spf_compact_spans: null pointer");
+  if (chunk < 1) return fail(SPF_ERR_INVALID_ARG, "spf_compact_spans: chunk must be >= 1 (got %d)", chunk);
+  if (n_tokens < 1 || n_tokens > 0x7fffffff)
+    return fail(SPF_ERR_INVALID_ARG, "spf_compact_spans: n_tokens must be in [1, 2^31) (got %lld)", (long long)n_tokens);
+  const int64_t n_chunks = ceil_div(n_tokens, chunk);
+  if (k < 1 || k > n_chunks)
+    return fail(SPF_ERR_INVALID_ARG, "spf_compact_spans: k must be in [1, n_chunks] (got k=%lld, n_chunks=%lld)", (long long)k,
+                (long long)n_chunks);
+  const int64_t blocks = 1 + ceil_div(k, kCompactThreads / 32);
+  compact_spans_kernel<<<(unsigned)blocks, kCompactThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      kept_chunks, (int)k, chunk, n_tokens, token_ids, char_start, char_end, out_ids, out_pos, out_tok_spans, out_char_spans,
+      out_counts);
+  SPF_CUDA_CHECK(cudaGetLastError());
+  return SPF_OK;
+}

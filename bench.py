@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
@@ -64,12 +64,17 @@ class ClockSampler:
         self.path = None
 
     def start(self):
+        """Starts nvidia-smi sampling every 50 ms and waits (up to 5 s) for its first line."""
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            deadline = time.time() + 5.0
+            while time.time() < deadline and os.path.getsize(self.path) == 0:
+                time.sleep(0.02)
+            self.skip = sum(1 for _ in open(self.path))      # lines written before the timed region
         except Exception:
             self.proc = None
 
@@ -85,7 +90,7 @@ class ClockSampler:
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         try:
-            for line in open(self.path):
+            for line in list(open(self.path))[getattr(self, "skip", 0):]:
                 parts = [p.strip() for p in line.split(",")]
                 if len(parts) < 7:
                     continue
@@ -106,6 +111,16 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------- oracle leg
+def pick_sample_layers(cfg, prompt, budget_s=15.0):
+    """How many layers the oracle can score in about `budget_s` seconds (times layer 0 to find out)."""
+    import oracle
+    from workloads import bf16_bits
+    t0 = time.perf_counter()
+    oracle.token_importance(bf16_bits(prompt.q[:1]), [bf16_bits(prompt.k[0])])
+    per_layer = time.perf_counter() - t0
+    return max(1, min(cfg.n_layers, int(budget_s / max(per_layer, 1e-3))))
+
+
 def oracle_sample(cfg, prompt, keep, sample_layers):
     """Times the oracle on `sample_layers` of the prompt's layers (all keys) plus the full selection and
     scales the scoring time to all layers.  Returns (tokens/s, seconds of CPU work, description)."""
@@ -146,19 +161,18 @@ def run_reference(args):
     cfg = CONFIGS[args.workload]
     prompt = make_prompt(cfg, 0, "cuda" if torch.cuda.is_available() else "cpu").to("cpu")
     keep = cfg.keep[0]
-    sample_layers = 1
-    for _ in range(max(0, min(args.warmup, 1))):
-        oracle_sample(cfg, prompt, keep, sample_layers)
+    steps = max(1, min(args.steps, 4))              # each step is seconds of CPU work
+    sample_layers = pick_sample_layers(cfg, prompt, budget_s=60.0 / steps)
     vals, secs, desc = [], 0.0, ""
-    for _ in range(args.steps):
+    for _ in range(steps):
         v, s, desc = oracle_sample(cfg, prompt, keep, sample_layers)
         vals.append(v)
         secs += s
     value = len(vals) / sum(1.0 / v for v in vals)
     cores = blas_threads()
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1e3 * cfg.lengths[0] / value, "higher_is_better": True,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": 1, "ms_per_step": 1e3 * cfg.lengths[0] / value, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": cfg.name, "n_tokens": cfg.lengths[0], "n_layers": cfg.n_layers,
                    "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
@@ -311,7 +325,7 @@ def run_ours(args):
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": args.e2e_steps}
     if world == 1 and not args.no_cpu_baseline:
         cpu_prompt = make_prompt(cfg, 0, dev).to("cpu")
-        v, secs, desc = oracle_sample(cfg, cpu_prompt, keep, 1)
+        v, secs, desc = oracle_sample(cfg, cpu_prompt, keep, pick_sample_layers(cfg, cpu_prompt))
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc,
                                 "cpu_seconds": secs}
     print(json.dumps(line), flush=True)

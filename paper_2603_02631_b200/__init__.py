@@ -2,22 +2,22 @@
 
 Thin Python binding over the C-ABI library ``libspf.so`` (see ``include/spf.h``).  Every step of the
 path runs in the library's CUDA kernels; PyTorch only provides device memory and streams.
-Importing this package loads the library and raises if it has not been built
-(``python -m paper_2603_02631_b200.build``): there is no CPU fallback.
+The first use of any name below loads the library and raises ImportError if it has not been built
+(``python -m paper_2603_02631_b200.build``): there is no CPU fallback.  Only the ``build`` submodule
+can be imported without the library, since it is what produces it.
 """
-from .binding import (  # noqa: F401
-    LIB_PATH,
-    SpfError,
-    Selection,
-    Selector,
-    lib,
-    spf_chunk_pool,
-    spf_compact_spans,
-    spf_keep_count,
-    spf_last_error,
-    spf_score,
-    spf_score_workspace_bytes,
-    spf_select_topk,
-    spf_status_string,
-    spf_version,
+import importlib
+
+_BINDING_NAMES = (
+    "LIB_PATH", "SpfError", "Selection", "Selector", "PromptBuffers", "lib", "spf_chunk_pool", "spf_compact_spans",
+    "spf_keep_count", "spf_last_error", "spf_score", "spf_score_workspace_bytes", "spf_select_topk",
+    "spf_status_string", "spf_version",
 )
+__all__ = list(_BINDING_NAMES) + ["binding"]
+
+
+def __getattr__(name):
+    if name == "binding" or name in _BINDING_NAMES:
+        binding = importlib.import_module(".binding", __name__)
+        return binding if name == "binding" else getattr(binding, name)
+    raise AttributeError(f"module {__name__!r} has no attribute {name!r}")

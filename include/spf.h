@@ -104,6 +104,34 @@ SPF_API int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int
                           size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
 
 /*
+ * spf_score without a caller-provided workspace (the paper has no counterpart; this exists for
+ * deployment reasons only).
+ *
+ * Some callers cannot hand over scratch memory because they cannot allocate any at the point where
+ * they score a prompt: a serving engine that has already given all free HBM to its KV-cache pool, a
+ * plugin that runs inside someone else's process under a no-allocation rule, or code on a path where
+ * the implicit device-wide synchronisation of cudaMalloc / cudaFree is not acceptable.  For them the
+ * library keeps SPF_STATIC_SCRATCH_BYTES of scratch in a static device array of its own (part of the
+ * loaded module: every GPU that loads the library holds it until the process exits) and this call
+ * uses it in place of `workspace`.  It computes exactly what spf_score computes with the general
+ * two-sweep kernels and calls no allocating routine.
+ *
+ *   - Arguments and results are those of spf_score; inputs and outputs are still the caller's.
+ *   - Prompts whose scratch need (spf_score_workspace_bytes gives an upper bound) exceeds
+ *     SPF_STATIC_SCRATCH_BYTES are rejected with SPF_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the array's device address (with that device current)
+ *     and caches it.  Make that first call outside any stream capture, with the device that owns
+ *     `cuda_stream` current.
+ *   - Every call on a device shares the one array, and the array keeps whatever the previous call
+ *     left in it.  The kernels write each scratch word before they read it, so nothing needs
+ *     clearing between calls; but two calls whose kernels overlap on the GPU (different streams,
+ *     no ordering) race on it and give wrong results.  Order them on one stream or with events.
+ */
+#define SPF_STATIC_SCRATCH_BYTES (8u << 20)
+SPF_API int32_t spf_score_static(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts,
+                                 void* cuda_stream);
+
+/*
  * Smoothing and chunk means (Appendix A.1.2; Algorithm 1, AvgPool1D and PartitionIntoChunks;
  * kernel size 13 and chunk size 32 / 128 in Appendix A.3):
  *     S[s]  = (1/w) * sum_{t = s - w/2}^{s + w/2} I[t]      terms outside [0, N) count as zero

@@ -44,6 +44,8 @@ def _load() -> ctypes.CDLL:
     dll.spf_score_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32]
     dll.spf_score.restype = i32
     dll.spf_score.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp, ctypes.c_size_t, vp, vp]
+    dll.spf_score_static.restype = i32
+    dll.spf_score_static.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp]
     dll.spf_chunk_pool.restype = i32
     dll.spf_chunk_pool.argtypes = [vp, i64, i32, i32, vp, vp]
     dll.spf_select_topk.restype = i32
@@ -158,6 +160,16 @@ def spf_score(prompts: Sequence[PromptBuffers], workspace: torch.Tensor, softmax
     _check(lib.spf_score(ctypes.byref(shape), arr, len(prompts), workspace.data_ptr(),
                          workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
            "spf_score")
+
+
+def spf_score_static(prompts: Sequence[PromptBuffers], softmax_scale: float = 0.0,
+                     stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_score for callers that cannot allocate: the library's built-in scratch array replaces the workspace.
+
+    Calls that overlap on the GPU share that array and race; keep them ordered on one stream.
+    """
+    shape, arr, _keep = _marshal(prompts, softmax_scale)
+    _check(lib.spf_score_static(ctypes.byref(shape), arr, len(prompts), _stream_ptr(stream)), "spf_score_static")
 
 
 def spf_chunk_pool(importance: torch.Tensor, pool_kernel: int, chunk: int, chunk_scores: torch.Tensor,

@@ -142,6 +142,72 @@ extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, 
   return SPF_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// spf_score_static: scoring for callers that cannot allocate.  The scratch is this file-scope device
+// array.  In host code its name is only a handle for the runtime, not a device address, so the
+// address is looked up once per device with cudaGetSymbolAddress and that pointer goes to the kernels.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[SPF_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+// Device address of g_static_scratch on the current device (looked up on the first call per device).
+int32_t static_scratch_ptr(void** out) {
+  int dev = 0;
+  SPF_CUDA_CHECK(cudaGetDevice(&dev));
+  static std::mutex mu;
+  static void* cached[64];
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev < 0 || dev >= 64) return fail(SPF_ERR_CUDA, "device ordinal %d out of range", dev);
+  if (cached[dev] == nullptr) {
+    void* ptr = nullptr;
+    SPF_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    if (ptr == nullptr) return fail(SPF_ERR_CUDA, "spf_score_static: the scratch array has no device address");
+    cached[dev] = ptr;
+  }
+  *out = cached[dev];
+  return SPF_OK;
+}
+
+}  // namespace
+
+extern "C" int32_t spf_score_static(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts,
+                                    void* cuda_stream) {
+  clear_error();
+  if (shape == nullptr || prompts == nullptr || n_prompts < 1)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score_static: null argument or n_prompts < 1");
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    const int32_t st = make_problem(shape, prompts[i], i, &p);
+    if (st != SPF_OK) return st;
+    const size_t need = score_mma_workspace_bytes(p);
+    if (need > (size_t)SPF_STATIC_SCRATCH_BYTES)
+      return fail(SPF_ERR_WORKSPACE,
+                  "spf_score_static: prompt %d needs %zu bytes of scratch, the built-in array holds %zu; use spf_score "
+                  "with a caller-provided workspace",
+                  i, need, (size_t)SPF_STATIC_SCRATCH_BYTES);
+  }
+  int sm_count = 0;
+  {
+    const int32_t st = device_sm_count(&sm_count);
+    if (st != SPF_OK) return st;
+  }
+  void* scratch = nullptr;
+  {
+    const int32_t st = static_scratch_ptr(&scratch);
+    if (st != SPF_OK) return st;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    make_problem(shape, prompts[i], i, &p);
+    // every kernel of this path writes the scratch words it later reads, so stale contents are harmless
+    const int32_t st = score_mma_launch(p, scratch, sm_count, stream);
+    if (st != SPF_OK) return st;
+  }
+  return SPF_OK;
+}
+
 extern "C" int64_t spf_keep_count(int64_t n_chunks, double keep_ratio) {
   if (n_chunks < 1) return 0;
   if (!(keep_ratio > 0.0)) return 1;

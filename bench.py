@@ -40,6 +40,8 @@ def parse_args():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--score-path", default="auto", choices=["auto", "general", "fused"],
+                    help="kernels behind spf_score: fused single-kernel path, general two-sweep path, or automatic")
     return ap.parse_args()
 
 
@@ -212,7 +214,23 @@ def run_ours(args):
                        chunk=cfg.chunk, pool_kernel=cfg.pool_kernel, device=dev)
     tokens_per_step = sum(cfg.lengths)
     stream = torch.cuda.current_stream()
-    launches_per_prompt = 7      # pack_q, score_lse, merge_lse, score_max, chunk_pool, select_topk, compact_spans
+    # which scoring kernels run: probe the fused path once on the first prompt (it refuses shapes it does not cover)
+    want = {"auto": 0, "general": 1, "fused": 2}[args.score_path]
+    fused = False
+    if want != 1:
+        spf.spf_set_score_path(2)
+        try:
+            p0 = prompts[0]
+            sel.run(p0.q, p0.k, p0.token_ids, p0.char_start, p0.char_end, keep)
+            fused = True
+        except spf.SpfError:
+            if want == 2:
+                raise
+    spf.spf_set_score_path(2 if fused else 1)
+    # kernels per prompt: fused: score_fused, chunk_pool, select_topk, compact_spans;
+    # general: pack_q, score_lse, merge_lse, score_max + the same three
+    launches_per_prompt = 4 if fused else 7
+    score_kernels = "score_fused_kernel" if fused else "pack_q + score_lse + merge_lse + score_max"
 
     def step():
         for p in prompts:
@@ -239,6 +257,9 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop()
     ms_total = t_start.elapsed_time(t_end)
+    status = int(sel.dev_status.item())
+    if status != 0:
+        raise RuntimeError(f"device status {status} ({spf.spf_status_string(status)}) after the timed region")
 
     # --- the scoring call on its own (same launches, events around spf_score only) --------------------
     score_ms = []
@@ -315,7 +336,7 @@ def run_ours(args):
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
         "gpu_launches": launches_per_prompt * n_prompts * args.steps,
-        "roofline": {"bound": "hbm", "kernel": "spf_score (pack_q + score_lse + merge_lse + score_max)",
+        "roofline": {"bound": "hbm", "kernel": f"spf_score ({score_kernels})",
                      "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                      "frac": achieved / peak, "traffic": None, "ms_per_launch": score_ms_avg,
                      "algorithmic_bytes": score_bytes},

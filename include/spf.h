@@ -48,7 +48,8 @@ typedef enum {
   SPF_ERR_UNSUPPORTED = -2, /* shape outside what the kernels cover (see spf_score)                 */
   SPF_ERR_WORKSPACE = -3,   /* workspace missing, misaligned or smaller than the size query says    */
   SPF_ERR_CUDA = -4,        /* a CUDA runtime call failed (no device, launch error)                 */
-  SPF_ERR_TIMEOUT = -5      /* device status only: a bounded wait inside a kernel ran out           */
+  SPF_ERR_TIMEOUT = -5,     /* device status only: a bounded wait inside a kernel ran out           */
+  SPF_ERR_RANGE = -6        /* device status only: a softmax row overflowed fp32 in the fused path  */
 } spf_status;
 
 /* Draft-model attention geometry shared by all prompts of a call. */
@@ -95,13 +96,25 @@ SPF_API size_t spf_score_workspace_bytes(const spf_shape* shape, const spf_promp
  * entry are irrelevant, contents on exit unspecified.  Calls that share a workspace must be ordered
  * on one stream.
  * `dev_status`: device int32, may be NULL.  Kernels store a negative spf_status there when a
- * device-side condition occurs (SPF_ERR_TIMEOUT from a bounded wait); they never trap.  The caller
- * zeroes it before the call and reads it after synchronising.
+ * device-side condition occurs (SPF_ERR_TIMEOUT from a bounded wait; SPF_ERR_RANGE when, in the fused
+ * path, some logit exceeds the sampled reference of its row by more than 2^187 and the row sum
+ * overflows -- the importance is then invalid and the call should be repeated on the general path);
+ * they never trap.  The caller zeroes it before the call and reads it after synchronising.
  * Errors: SPF_ERR_INVALID_ARG, SPF_ERR_UNSUPPORTED (d not 64/128, Hq % Hkv != 0, m > 32,
  * G * roundup(m,8) > 64, L > 128), SPF_ERR_WORKSPACE, SPF_ERR_CUDA.
  */
 SPF_API int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace,
                           size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * Chooses the kernels behind spf_score, process-wide: 0 = automatic (the fused single-kernel path when
+ * the shape allows it, else the general two-sweep path), 1 = always the general path, 2 = always the
+ * fused path (spf_score then returns SPF_ERR_UNSUPPORTED for shapes outside it: G not in {1,2,4,8},
+ * more than 64 layers, or a prompt too long for the per-CTA state).  Both compute the same function
+ * (Appendix A.1.1).  Meant for tests and measurements.  Returns the previous setting; an invalid value
+ * changes nothing.
+ */
+SPF_API int32_t spf_set_score_path(int32_t path);
 
 /*
  * spf_score without a caller-provided workspace (the paper has no counterpart; this exists for

@@ -44,6 +44,8 @@ def _load() -> ctypes.CDLL:
     dll.spf_score_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32]
     dll.spf_score.restype = i32
     dll.spf_score.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp, ctypes.c_size_t, vp, vp]
+    dll.spf_set_score_path.restype = i32
+    dll.spf_set_score_path.argtypes = [i32]
     dll.spf_score_static.restype = i32
     dll.spf_score_static.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp]
     dll.spf_chunk_pool.restype = i32
@@ -160,6 +162,11 @@ def spf_score(prompts: Sequence[PromptBuffers], workspace: torch.Tensor, softmax
     _check(lib.spf_score(ctypes.byref(shape), arr, len(prompts), workspace.data_ptr(),
                          workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
            "spf_score")
+
+
+def spf_set_score_path(path: int) -> int:
+    """0 automatic, 1 general two-sweep path, 2 fused path; returns the previous setting."""
+    return int(lib.spf_set_score_path(path))
 
 
 def spf_score_static(prompts: Sequence[PromptBuffers], softmax_scale: float = 0.0,

@@ -1,4 +1,5 @@
 // Host side of the C ABI: argument validation, error text, dispatch of spf_score.
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -10,6 +11,7 @@ namespace spf {
 namespace {
 
 thread_local char g_error[512] = "";
+std::atomic<int> g_score_path{0};  // 0 automatic, 1 general two-sweep path, 2 fused path
 
 // Builds the per-prompt problem description; returns a status and leaves the reason in the error text.
 int32_t make_problem(const spf_shape* shape, const spf_prompt& pr, int32_t index, ScoreProblem* out) {
@@ -104,7 +106,7 @@ extern "C" size_t spf_score_workspace_bytes(const spf_shape* shape, const spf_pr
   for (int32_t i = 0; i < n_prompts; ++i) {
     ScoreProblem p;
     if (make_problem(shape, prompts[i], i, &p) != SPF_OK) return 0;
-    need = std::max(need, score_mma_workspace_bytes(p));
+    need = std::max(need, std::max(score_mma_workspace_bytes(p), score_fused_workspace_bytes(p)));
   }
   return need;
 }
@@ -112,7 +114,6 @@ extern "C" size_t spf_score_workspace_bytes(const spf_shape* shape, const spf_pr
 extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace,
                              size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
   clear_error();
-  (void)dev_status;  // the two-sweep path has no device-side wait that could run out
   if (shape == nullptr || prompts == nullptr || n_prompts < 1)
     return fail(SPF_ERR_INVALID_ARG, "spf_score: null argument or n_prompts < 1");
   // validate everything before the first launch
@@ -121,7 +122,7 @@ extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, 
     ScoreProblem p;
     const int32_t st = make_problem(shape, prompts[i], i, &p);
     if (st != SPF_OK) return st;
-    need = std::max(need, score_mma_workspace_bytes(p));
+    need = std::max(need, std::max(score_mma_workspace_bytes(p), score_fused_workspace_bytes(p)));
   }
   if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
     return fail(SPF_ERR_WORKSPACE, "spf_score: workspace is null or not 256-byte aligned");
@@ -136,10 +137,18 @@ extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, 
   for (int32_t i = 0; i < n_prompts; ++i) {
     ScoreProblem p;
     make_problem(shape, prompts[i], i, &p);
-    const int32_t st = score_mma_launch(p, workspace, sm_count, stream);
+    const int path = g_score_path.load(std::memory_order_relaxed);
+    const bool fused = path == 2 || (path == 0 && score_fused_supported(p, sm_count));
+    const int32_t st = fused ? score_fused_launch(p, workspace, sm_count, dev_status, stream)
+                             : score_mma_launch(p, workspace, sm_count, stream);
     if (st != SPF_OK) return st;
   }
   return SPF_OK;
+}
+
+extern "C" int32_t spf_set_score_path(int32_t path) {
+  if (path < 0 || path > 2) return g_score_path.load(std::memory_order_relaxed);
+  return g_score_path.exchange(path, std::memory_order_relaxed);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -224,6 +233,7 @@ extern "C" const char* spf_status_string(int32_t status) {
     case SPF_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case SPF_ERR_CUDA: return "CUDA runtime error";
     case SPF_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case SPF_ERR_RANGE: return "a softmax row overflowed fp32 in the fused path";
     default: return "unknown status";
   }
 }

@@ -1,0 +1,886 @@
+// Token-importance scoring, fused path: ONE persistent kernel that reads the key cache once from HBM.
+//
+// Why two visits per key tile.  The max over (layer, head) is taken over softmax PROBABILITIES, so a
+// logit can only be compared across heads after its row's log-sum-exp is known, and that needs all N
+// keys of the row.  Each (layer, kv-head) slab of keys is therefore visited twice:
+//   visit 1 ("sum")  accumulates  sum_s exp2(c * q.k - ref)  per query row;
+//   visit 2 ("max")  folds  max_{l,h} (q.k - lse/c)  into a running maximum per (lookahead i, key s).
+// The kernel software-pipelines the two visits by `lag` slabs: while slab t streams in from HBM for
+// visit 1, slab t - lag is read again for visit 2 -- by the same CTA that read it a few microseconds
+// earlier, so the second read is served by L2.
+//
+// Work split.  The grid is persistent (one CTA per SM).  CTA b owns key tiles b, b + grid, ... (128
+// keys each) of EVERY slab, so its running maxima for those keys stay in its shared memory for the
+// whole kernel and the importance of a key is written exactly once, at the end.
+//
+// One tile = one tcgen05 MMA group: A = 128 keys x d (shared memory, TMA, 128-byte swizzle),
+// B = the slab's query rows x d (row j = i * G + g: lookahead i, head g of the GQA group), D = fp32
+// [128 keys x NCOLS rows] in tensor memory.  Keys are TMEM lanes, so an epilogue thread owns one key
+// and sees all query rows of it: the max over heads is in-thread, and the sum over keys is kept
+// per thread and reduced across threads only once per slab.
+//
+// Folded offsets.  An extra 16-wide MMA step multiplies a constant tile of ones (key side) with a
+// small tile holding, per query row, an offset split into three bf16 terms.  Visit 1 uses
+// -ref/c (a reference logit, so that exp2 cannot overflow), visit 2 uses -lse/c.  The subtraction
+// thus happens in the tensor core's fp32 accumulator and costs no ALU instruction per logit.
+// The reference of a row is the largest logit among a few sample keys of the CTA plus a margin of 60
+// (base-2 units): sums stay finite unless some key beats the samples by more than 2^187, in which
+// case the row's sum becomes inf and SPF_ERR_RANGE is reported.
+//
+// Cross-CTA step.  After visit 1 of a slab every CTA publishes its partial (ref, sum) per row; the
+// CTA that arrives last merges them into lse2[slab][row] and raises a flag that the visit-2 side of
+// every CTA waits for.  Because visit 1 never waits on another CTA and all CTAs are co-resident,
+// the flags always get raised.
+//
+// Every wait in this file is bounded: on expiry the kernel records SPF_ERR_TIMEOUT, drains and
+// returns normally.
+#include <cuda.h>
+
+#include <algorithm>
+#include <mutex>
+
+#include "common.cuh"
+#include "score.cuh"
+
+namespace spf {
+namespace {
+
+constexpr int kTileKeys = 128;
+constexpr int kThreads = 384;          // warp 0 TMA, 1 MMA, 2 control, 3 idle, 4..11 epilogue
+constexpr int kEpiWarps = 8;
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kQStages = 3;
+constexpr int kTmemStages = 4;
+constexpr int kRefSlots = 8;
+constexpr int kMaxSamples = 4;
+constexpr float kRefMargin = 60.f;     // base-2 units added to the sampled reference logit
+constexpr unsigned long long kTimeoutNs = 2000000000ull;
+constexpr int kSubTileBytes = kTileKeys * 128;  // 128 keys x 64 bf16, one swizzle-128B tile
+constexpr int kQSubTileBytes = 64 * 128;        // up to 64 query rows x 64 bf16
+
+struct FusedMaps {
+  CUtensorMap q;                      // (d, g, i, slab) view of the query tensor
+  CUtensorMap k[kFusedMaxLayers];     // (d, key, kv-head) view of each layer's key cache
+};
+
+struct FusedArgs {
+  const __nv_bfloat16* k_layers[kFusedMaxLayers];
+  const __nv_bfloat16* q;
+  int64_t n_tokens, stride_head, stride_tok;
+  int n_layers, n_kv_heads, n_lookahead, n_tiles, tiles_per_cta_max, lag, k_stages;
+  float c, inv_c;
+  float2* partial;        // [slab][cta][NCOLS] (ref, sum)
+  float* lse2;            // [slab][NCOLS]
+  unsigned* counters;     // [slab] arrivals of visit 1
+  unsigned* ready;        // [slab] 1 once lse2[slab] is final
+  float* lse_out;         // optional [L][Hq][m], natural log
+  float* importance;      // [N]
+  int32_t* dev_status;    // optional
+};
+
+// ---------------------------------------------------------------------------------------------- PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long global_timer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+struct Abort {
+  volatile int* flag;      // shared: set once any wait of this CTA ran out
+  int32_t* dev_status;     // global, may be null
+};
+
+__device__ __noinline__ void record_timeout(const Abort& ab) {
+  *ab.flag = 1;
+  if (ab.dev_status != nullptr) atomicCAS(ab.dev_status, 0, (int32_t)SPF_ERR_TIMEOUT);
+}
+
+// Waits for the phase with the given parity; false if the CTA is aborting or the wait ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab) {
+  if (mbar_try_wait(bar, parity)) return true;
+  unsigned long long t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*ab.flag) return false;
+      const unsigned long long now = global_timer();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kTimeoutNs) {
+        record_timeout(ab);
+        return false;
+      }
+    }
+  }
+}
+
+// Warp-collective form: every lane waits, and all lanes agree on the outcome (a timeout seen by one
+// lane only must not split the warp in front of .aligned instructions).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const Abort& ab) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, ab));
+}
+
+// Waits until *flag (global) becomes non-zero, with acquire semantics.
+__device__ __forceinline__ bool flag_wait(const unsigned* flag, const Abort& ab) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v != 0u) return true;
+    if ((it & 15u) == 15u) {
+      if (*ab.flag) return false;
+      const unsigned long long now = global_timer();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kTimeoutNs) {
+        record_timeout(ab);
+        return false;
+      }
+      __nanosleep(100);
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);   // start address / 16
+  d |= (uint64_t)1 << 16;                    // leading byte offset (not used by swizzled K-major operands)
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset: 8 rows x 128 bytes
+  d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileKeys >> 4) << 24);
+}
+
+template <int N>
+__device__ __forceinline__ void tmem_load(uint32_t taddr, float (&v)[N]);
+
+template <>
+__device__ __forceinline__ void tmem_load<8>(uint32_t taddr, float (&v)[8]) {
+  uint32_t r[8];
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+template <>
+__device__ __forceinline__ void tmem_load<16>(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+template <>
+__device__ __forceinline__ void tmem_load<32>(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,"
+      "%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Byte offset of element (row, col) of a [rows x 64] bf16 tile stored with the 128-byte swizzle.
+__device__ __forceinline__ uint32_t swz128(int row, int col) {
+  const int byte = col * 2;
+  return (uint32_t)(row * 128 + ((((byte >> 4) ^ (row & 7)) << 4) | (byte & 15)));
+}
+
+__device__ __forceinline__ unsigned short bf16_bits_rn(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
+__device__ __forceinline__ float bf16_value(unsigned short b) { return __uint_as_float((uint32_t)b << 16); }
+
+// Writes value v (split into three bf16 terms) into row `row`, step `step` of the offsets tile and
+// returns the sum of the three terms, i.e. the offset the tensor core will add.
+__device__ __forceinline__ float write_offset(unsigned char* tile, int row, int step, float v) {
+  const unsigned short t0 = bf16_bits_rn(v);
+  const float r1 = v - bf16_value(t0);
+  const unsigned short t1 = bf16_bits_rn(r1);
+  const float r2 = r1 - bf16_value(t1);
+  const unsigned short t2 = bf16_bits_rn(r2);
+  unsigned short* dst = reinterpret_cast<unsigned short*>(tile + swz128(row, step * 16));
+  dst[0] = t0;
+  dst[1] = t1;
+  dst[2] = t2;
+  return bf16_value(t0) + bf16_value(t1) + bf16_value(t2);
+}
+
+// ---------------------------------------------------------------------------------------------- layout
+struct SmemLayout {
+  uint32_t k_off, q_off, ones_off, offs_off, amax_off, ref_off, red_off, merge_off, bar_off, misc_off, total;
+};
+
+__host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, int k_stages, int tiles_per_cta_max) {
+  SmemLayout s;
+  uint32_t o = 0;
+  s.k_off = o;        o += (uint32_t)k_stages * (d / 64) * kSubTileBytes;
+  s.q_off = o;        o += (uint32_t)kQStages * (d / 64) * kQSubTileBytes;
+  s.ones_off = o;     o += kSubTileBytes;
+  s.offs_off = o;     o += kQSubTileBytes;
+  s.amax_off = o;     o += (uint32_t)tiles_per_cta_max * (ncols / group) * kTileKeys * 4;
+  s.ref_off = o;      o += kRefSlots * 64 * 4;
+  s.red_off = o;      o += 4 * 64 * 4;
+  s.merge_off = o;    o += kEpiThreads * 8;
+  s.bar_off = o;      o += 64 * 8;
+  s.misc_off = o;     o += 64;
+  s.total = o;
+  return s;
+}
+
+// mbarrier addresses inside the barrier block
+struct Bars {
+  uint32_t base;
+  int k_stages;
+  __device__ uint32_t k_full(int s) const { return base + 8u * s; }
+  __device__ uint32_t k_empty(int s) const { return base + 8u * (k_stages + s); }
+  __device__ uint32_t q_full(int s) const { return base + 8u * (2 * k_stages + s); }
+  __device__ uint32_t q_empty(int s) const { return base + 8u * (2 * k_stages + kQStages + s); }
+  __device__ uint32_t t_full(int s) const { return base + 8u * (2 * k_stages + 2 * kQStages + s); }
+  __device__ uint32_t t_empty(int s) const { return base + 8u * (2 * k_stages + 2 * kQStages + kTmemStages + s); }
+  __device__ uint32_t o_ready(int x) const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + x); }
+  __device__ uint32_t o_free(int x) const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 4 + x); }
+  __device__ uint32_t epi_sync() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 8); }
+  __device__ uint32_t mma_done() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 9); }
+};
+// 2 * 8 + 2 * 3 + 2 * 4 + 10 = 40 barriers at most; the block has room for 64.
+
+struct Ring {
+  int stage = 0;
+  uint32_t phase = 0;
+  int n;
+  __device__ explicit Ring(int n_) : n(n_) {}
+  __device__ void advance() {
+    if (++stage == n) {
+      stage = 0;
+      phase ^= 1u;
+    }
+  }
+};
+
+// Barrier among the eight epilogue warps, with a bounded wait (an mbarrier with one arrival per warp).
+struct EpiSync {
+  uint32_t bar;
+  uint32_t phase = 0;
+  __device__ bool sync(int lane, const Abort& ab) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+    const bool ok = mbar_wait_warp(bar, phase, ab);
+    phase ^= 1u;
+    return ok;
+  }
+};
+
+// ---------------------------------------------------------------------------------------------- kernel
+template <int D, int NCOLS, int G>
+__global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_constant__ FusedMaps maps,
+                                                                   const __grid_constant__ FusedArgs a) {
+  constexpr int CH = NCOLS / 2;          // query rows (TMEM columns) per epilogue thread
+  constexpr int NI = NCOLS / G;          // lookahead slots per key in the running-max array
+  constexpr int KSUB = D / 64;           // 64-wide sub-tiles per key tile
+  static_assert(CH % G == 0, "a thread must own whole GQA groups");
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const SmemLayout lay = smem_layout(D, NCOLS, G, a.k_stages, a.tiles_per_cta_max);
+  unsigned char* k_tiles = smem + lay.k_off;
+  unsigned char* q_tiles = smem + lay.q_off;
+  unsigned char* ones_tile = smem + lay.ones_off;
+  unsigned char* offs_tile = smem + lay.offs_off;
+  float* amax = reinterpret_cast<float*>(smem + lay.amax_off);       // [local tile][NI][128]
+  float* ref_slots = reinterpret_cast<float*>(smem + lay.ref_off);   // [kRefSlots][64]
+  float* red = reinterpret_cast<float*>(smem + lay.red_off);         // [4 quadrants][64]
+  float2* merge_buf = reinterpret_cast<float2*>(smem + lay.merge_off);
+  volatile int* misc = reinterpret_cast<volatile int*>(smem + lay.misc_off);  // [0] abort, [1] tmem base, [2] is_last
+  const Bars bars{smem_u32(smem + lay.bar_off), a.k_stages};
+  const Abort ab{misc, a.dev_status};
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x, n_cta = gridDim.x;
+  const int n_slabs = a.n_layers * a.n_kv_heads;
+  const int my_tiles = (a.n_tiles - cta + n_cta - 1) / n_cta;      // tiles cta, cta + n_cta, ...
+  const int rows_real = G * a.n_lookahead;                         // query rows that exist (<= NCOLS)
+
+  // ------------------------------------------------------------------ set-up
+  if (threadIdx.x == 0) {
+    misc[0] = 0;
+    misc[1] = 0;
+    misc[2] = 0;
+    for (int s = 0; s < a.k_stages; ++s) {
+      mbar_init(bars.k_full(s), 1);
+      mbar_init(bars.k_empty(s), 1);
+    }
+    for (int s = 0; s < kQStages; ++s) {
+      mbar_init(bars.q_full(s), 1);
+      mbar_init(bars.q_empty(s), 1);
+    }
+    for (int s = 0; s < kTmemStages; ++s) {
+      mbar_init(bars.t_full(s), 1);
+      mbar_init(bars.t_empty(s), kEpiWarps);
+    }
+    for (int x = 0; x < 4; ++x) {
+      mbar_init(bars.o_ready(x), 1);
+      mbar_init(bars.o_free(x), 1);
+    }
+    mbar_init(bars.epi_sync(), kEpiWarps);
+    mbar_init(bars.mma_done(), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // zero the query stages (rows the TMA box does not cover must read as zero), the offsets tile and the
+  // constant tile; the constant tile then gets ones in the first three columns of each 16-wide step
+  for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kQStages * KSUB * kQSubTileBytes; i += kThreads * 16)
+    *reinterpret_cast<uint4*>(q_tiles + i) = make_uint4(0, 0, 0, 0);
+  for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kQSubTileBytes; i += kThreads * 16)
+    *reinterpret_cast<uint4*>(offs_tile + i) = make_uint4(0, 0, 0, 0);
+  for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kSubTileBytes; i += kThreads * 16)
+    *reinterpret_cast<uint4*>(ones_tile + i) = make_uint4(0, 0, 0, 0);
+  __syncthreads();
+  for (int i = threadIdx.x; i < kTileKeys * 4 * 3; i += kThreads) {
+    const int row = i / 12, step = (i % 12) / 3, t = i % 3;
+    *reinterpret_cast<unsigned short*>(ones_tile + swz128(row, step * 16 + t)) = 0x3F80;  // bf16 1.0
+  }
+  for (int i = threadIdx.x; i < my_tiles * NI * kTileKeys; i += kThreads) amax[i] = -INFINITY;
+  fence_async_smem();
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)&misc[1])),
+                 "r"(kTmemStages * NCOLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = (uint32_t)misc[1];
+
+  // ------------------------------------------------------------------ roles
+  if (warp == 0) {
+    // ===== TMA producer: one query tile per visit, then the CTA's key tiles of the slab =====
+    if (lane == 0) {
+      Ring kr(a.k_stages), qr(kQStages);
+      bool ok = true;
+      for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
+        for (int visit = 0; ok && visit < 2; ++visit) {
+          const int slab = visit == 0 ? t : t - a.lag;
+          if (slab < 0 || slab >= n_slabs) continue;
+          const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
+          if (!(ok = mbar_wait(bars.q_empty(qr.stage), qr.phase ^ 1u, ab))) break;
+          mbar_expect_tx(bars.q_full(qr.stage), (uint32_t)(KSUB * rows_real * 128));
+          for (int h = 0; h < KSUB; ++h)
+            tma_load_4d(smem_u32(q_tiles + (qr.stage * KSUB + h) * kQSubTileBytes), &maps.q, h * 64, 0, 0, slab,
+                        bars.q_full(qr.stage));
+          qr.advance();
+          for (int lt = 0; lt < my_tiles; ++lt) {
+            if (!(ok = mbar_wait(bars.k_empty(kr.stage), kr.phase ^ 1u, ab))) break;
+            mbar_expect_tx(bars.k_full(kr.stage), (uint32_t)(KSUB * kSubTileBytes));
+            const int key0 = (cta + lt * n_cta) * kTileKeys;
+            for (int h = 0; h < KSUB; ++h)
+              tma_load_3d(smem_u32(k_tiles + (kr.stage * KSUB + h) * kSubTileBytes), &maps.k[layer], h * 64, key0, hk,
+                          bars.k_full(kr.stage));
+            kr.advance();
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===== MMA issuer =====
+    if (lane == 0) {
+      Ring kr(a.k_stages), qr(kQStages), tr(kTmemStages);
+      constexpr uint32_t idesc = instr_desc(NCOLS);
+      const uint64_t ones_desc = smem_desc(smem_u32(ones_tile));
+      const uint64_t offs_desc = smem_desc(smem_u32(offs_tile));
+      bool ok = true;
+      for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
+        for (int visit = 0; ok && visit < 2; ++visit) {
+          const int slab = visit == 0 ? t : t - a.lag;
+          if (slab < 0 || slab >= n_slabs) continue;
+          const int x = visit * 2 + (slab & 1);                 // which 16-wide step of the offsets tile
+          if (!(ok = mbar_wait(bars.q_full(qr.stage), qr.phase, ab))) break;
+          if (!(ok = mbar_wait(bars.o_ready(x), (uint32_t)(slab >> 1) & 1u, ab))) break;
+          for (int lt = 0; lt < my_tiles; ++lt) {
+            if (!(ok = mbar_wait(bars.k_full(kr.stage), kr.phase, ab))) break;
+            if (!(ok = mbar_wait(bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(tr.stage * NCOLS);
+#pragma unroll
+            for (int h = 0; h < KSUB; ++h) {
+              const uint64_t ad = smem_desc(smem_u32(k_tiles + (kr.stage * KSUB + h) * kSubTileBytes));
+              const uint64_t bd = smem_desc(smem_u32(q_tiles + (qr.stage * KSUB + h) * kQSubTileBytes));
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks) tc_mma(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
+            }
+            tc_mma(d_tmem, ones_desc + 2u * x, offs_desc + 2u * x, idesc, 1u);
+            tc_commit(bars.k_empty(kr.stage));
+            tc_commit(bars.t_full(tr.stage));
+            kr.advance();
+            tr.advance();
+          }
+          if (!ok) break;
+          tc_commit(bars.q_empty(qr.stage));
+          tc_commit(bars.o_free(x));
+          qr.advance();
+        }
+      }
+      // leave only after everything issued has completed and signalled its barriers
+      if (ok) {
+        tc_commit(bars.mma_done());
+        mbar_wait(bars.mma_done(), 0u, ab);
+      }
+    }
+  } else if (warp == 2) {
+    // ===== control warp: per-row offsets for the extra MMA step; lane handles rows lane and lane + 32 =====
+    bool ok = true;
+    const int n_samples = min(my_tiles, kMaxSamples);
+    for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
+      for (int visit = 0; ok && visit < 2; ++visit) {
+        const int slab = visit == 0 ? t : t - a.lag;
+        if (slab < 0 || slab >= n_slabs) continue;
+        const int x = visit * 2 + (slab & 1);
+        const int use = slab >> 1;                              // how often step x was written before
+        if (use > 0) {
+          if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
+        }
+        float value[2] = {0.f, 0.f};                            // offsets of rows lane, lane + 32 in q.k units
+        if (visit == 0) {
+          // reference logit: max over a few sample keys of this CTA's range, plus a margin
+          const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
+          const __nv_bfloat16* kslab = a.k_layers[layer] + hk * a.stride_head;
+          float best[2] = {-INFINITY, -INFINITY};
+          for (int sidx = 0; sidx < n_samples; ++sidx) {
+            const int64_t key = (int64_t)(cta + sidx * n_cta) * kTileKeys;
+            const uint4* krow = reinterpret_cast<const uint4*>(kslab + key * a.stride_tok);
+            float dot[2] = {0.f, 0.f};
+            for (int ch = 0; ch < D / 8; ++ch) {
+              const uint4 kv = __ldg(krow + ch);
+              const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv);
+#pragma unroll
+              for (int r = 0; r < 2; ++r) {
+                const int row = lane + 32 * r;
+                if (row < rows_real) {
+                  const int i = row / G, g = row % G;
+                  const uint4 qv = __ldg(reinterpret_cast<const uint4*>(
+                                             a.q + (((int64_t)slab * G + g) * a.n_lookahead + i) * D) + ch);
+                  const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv);
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    const float2 kf = __bfloat1622float2(k2[e]), qf = __bfloat1622float2(q2[e]);
+                    dot[r] = fmaf(kf.x, qf.x, fmaf(kf.y, qf.y, dot[r]));
+                  }
+                }
+              }
+            }
+            best[0] = fmaxf(best[0], dot[0]);
+            best[1] = fmaxf(best[1], dot[1]);
+          }
+#pragma unroll
+          for (int r = 0; r < 2; ++r)
+            if (lane + 32 * r < rows_real) value[r] = -(best[r] + kRefMargin * a.inv_c);
+        } else {
+          if (!(ok = __all_sync(0xffffffffu, flag_wait(a.ready + slab, ab)))) break;
+#pragma unroll
+          for (int r = 0; r < 2; ++r)
+            if (lane + 32 * r < rows_real) value[r] = -__ldcg(a.lse2 + (int64_t)slab * NCOLS + lane + 32 * r) * a.inv_c;
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const int row = lane + 32 * r;
+          if (row < NCOLS) {
+            const float seen = write_offset(offs_tile, row, x, value[r]);
+            if (visit == 0) ref_slots[(slab % kRefSlots) * 64 + row] = -seen * a.c;   // reference in base-2 units
+          }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars.o_ready(x));
+      }
+    }
+  } else if (warp >= 4) {
+    // ===== epilogue: 8 warps; warp % 4 picks the TMEM lane quadrant (keys), warps 4-7 / 8-11 the column half =====
+    const int quad = warp & 3;
+    const int hh = (warp - 4) >> 2;
+    const int et = threadIdx.x - 128;                           // 0..255 among epilogue threads
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    Ring tr(kTmemStages);
+    EpiSync es{bars.epi_sync()};
+    bool ok = true;
+    for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
+      for (int visit = 0; ok && visit < 2; ++visit) {
+        const int slab = visit == 0 ? t : t - a.lag;
+        if (slab < 0 || slab >= n_slabs) continue;
+        if (visit == 0) {
+          // ---------------- visit 1: per-thread sums of exp2 over the thread's keys ----------------
+          float sum[CH];
+#pragma unroll
+          for (int j = 0; j < CH; ++j) sum[j] = 0.f;
+          for (int lt = 0; lt < my_tiles; ++lt) {
+            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+            tc_fence_after();
+            float v[CH];
+            tmem_load<CH>(tmem_base + lane_addr + (uint32_t)(tr.stage * NCOLS + hh * CH), v);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
+            tr.advance();
+            const int64_t key = (int64_t)(cta + lt * n_cta) * kTileKeys + quad * 32 + lane;
+            if (key < a.n_tokens) {
+#pragma unroll
+              for (int j = 0; j < CH; ++j) sum[j] += fast_exp2(v[j] * a.c);
+            }
+          }
+          if (!ok) break;
+          // reduce over the 32 keys of the warp: transposing butterfly while more than one column is
+          // left per thread, plain butterfly afterwards
+          {
+            int width = CH;
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) {
+              if (width > 1) {
+                width >>= 1;
+                const bool upper = (lane & off) != 0;
+#pragma unroll
+                for (int j = 0; j < CH / 2; ++j) {
+                  if (j < width) {
+                    const float send = upper ? sum[j] : sum[j + width];
+                    const float keep = upper ? sum[j + width] : sum[j];
+                    sum[j] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+                  }
+                }
+              } else {
+                sum[0] += __shfl_xor_sync(0xffffffffu, sum[0], off);
+              }
+            }
+          }
+          // the lane now holds the warp total of column hh * CH + lane / (32 / CH)
+          constexpr int kLanesPerCol = 32 / CH;
+          if (lane % kLanesPerCol == 0) red[quad * 64 + hh * CH + lane / kLanesPerCol] = sum[0];
+          if (!(ok = es.sync(lane, ab))) break;
+          if (et < NCOLS) {
+            const float total = red[et] + red[64 + et] + red[128 + et] + red[192 + et];
+            const float ref = ref_slots[(slab % kRefSlots) * 64 + et];
+            __stcg(a.partial + ((int64_t)slab * n_cta + cta) * NCOLS + et, make_float2(ref, total));
+            __threadfence();
+          }
+          if (!(ok = es.sync(lane, ab))) break;
+          if (et == 0) {
+            const unsigned old = atomicAdd(a.counters + slab, 1u);
+            misc[2] = old == (unsigned)(n_cta - 1);
+          }
+          if (!(ok = es.sync(lane, ab))) break;
+          if (misc[2]) {
+            // last CTA to finish visit 1 of this slab: merge all partials into lse2[slab][:]
+            __threadfence();
+            constexpr int kSubsets = kEpiThreads / NCOLS;
+            const int col = et % NCOLS, sub = et / NCOLS;
+            float m = -INFINITY, z = 0.f;
+            for (int b = sub; b < n_cta; b += kSubsets) {
+              const float2 p = __ldcg(a.partial + ((int64_t)slab * n_cta + b) * NCOLS + col);
+              const float v = p.x + log2f(p.y);                // log2 of this CTA's share of the row sum
+              const float mm = fmaxf(m, v);
+              z = z * exp2f(m - mm) + exp2f(v - mm);
+              m = mm;
+            }
+            merge_buf[et] = make_float2(m, z);
+            if (!(ok = es.sync(lane, ab))) break;
+            if (et < NCOLS) {
+              float mm = -INFINITY;
+              for (int s2 = 0; s2 < kSubsets; ++s2) mm = fmaxf(mm, merge_buf[s2 * NCOLS + et].x);
+              float zz = 0.f;
+              for (int s2 = 0; s2 < kSubsets; ++s2) {
+                const float2 p = merge_buf[s2 * NCOLS + et];
+                if (p.x > -INFINITY) zz += p.y * exp2f(p.x - mm);
+              }
+              const float lse2 = mm + log2f(zz);
+              __stcg(a.lse2 + (int64_t)slab * NCOLS + et, lse2);
+              const int i = et / G, g = et % G;
+              if (a.lse_out != nullptr && i < a.n_lookahead)
+                a.lse_out[((int64_t)slab * G + g) * a.n_lookahead + i] = lse2 * kLn2;
+              if (et < rows_real && !(lse2 > -INFINITY && lse2 < INFINITY) && a.dev_status != nullptr)
+                atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
+              __threadfence();
+            }
+            if (!(ok = es.sync(lane, ab))) break;
+            if (et == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.ready + slab), "r"(1u) : "memory");
+          }
+        } else {
+          // ---------------- visit 2: running max over (layer, head) of q.k - lse/c ----------------
+          for (int lt = 0; lt < my_tiles; ++lt) {
+            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+            tc_fence_after();
+            float v[CH];
+            tmem_load<CH>(tmem_base + lane_addr + (uint32_t)(tr.stage * NCOLS + hh * CH), v);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
+            tr.advance();
+            float* slot = amax + ((int64_t)lt * NI + hh * (CH / G)) * kTileKeys + quad * 32 + lane;
+#pragma unroll
+            for (int ii = 0; ii < CH / G; ++ii) {
+              float mx = v[ii * G];
+#pragma unroll
+              for (int g = 1; g < G; ++g) mx = fmaxf(mx, v[ii * G + g]);
+              if (hh * (CH / G) + ii < a.n_lookahead) slot[ii * kTileKeys] = fmaxf(slot[ii * kTileKeys], mx);
+            }
+          }
+        }
+      }
+    }
+    // ---------------- importance: mean over lookahead of exp2(c * running max) ----------------
+    if (ok) ok = es.sync(lane, ab);
+    if (ok && misc[0] == 0) {
+      const float inv_m = 1.f / (float)a.n_lookahead;
+      for (int idx = et; idx < my_tiles * kTileKeys; idx += kEpiThreads) {
+        const int lt = idx / kTileKeys, kk = idx % kTileKeys;
+        const int64_t key = (int64_t)(cta + lt * n_cta) * kTileKeys + kk;
+        if (key < a.n_tokens) {
+          float s = 0.f;
+          for (int i = 0; i < a.n_lookahead; ++i) s += fast_exp2(amax[((int64_t)lt * NI + i) * kTileKeys + kk] * a.c);
+          a.importance[key] = s * inv_m;
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (misc[0] != 0) {
+    // a wait ran out somewhere: give copies and MMAs still in flight time to land before TMEM goes away
+    const unsigned long long t0 = global_timer();
+    while (global_timer() - t0 < 2000000ull) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemStages * NCOLS) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static std::once_flag once;
+  static EncodeTiledFn fn = nullptr;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult res;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &res) == cudaSuccess &&
+        res == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+struct FusedPlan {
+  bool ok = false;
+  int ncols = 0, k_stages = 0, tiles_per_cta_max = 0, n_cta = 0, n_tiles = 0;
+  SmemLayout lay{};
+};
+
+constexpr int kSmemBudget = 227 * 1024 - 1024;   // dynamic shared memory we may ask for, minus alignment slack
+
+FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
+  FusedPlan pl;
+  const int g = p.group;
+  if (!(g == 1 || g == 2 || g == 4 || g == 8)) return pl;
+  if (p.n_layers > kFusedMaxLayers) return pl;
+  const int rows = g * p.n_lookahead;
+  if (rows > 64) return pl;
+  if (p.n_tokens > (int64_t)1 << 30) return pl;
+  pl.ncols = rows <= 16 ? 16 : rows <= 32 ? 32 : 64;
+  pl.n_tiles = (int)ceil_div(p.n_tokens, kTileKeys);
+  pl.n_cta = std::min(std::min(sm_count, kFusedMaxCtas), pl.n_tiles);
+  pl.tiles_per_cta_max = (int)ceil_div(pl.n_tiles, pl.n_cta);
+  for (int ks = 8; ks >= 3; --ks) {
+    const SmemLayout lay = smem_layout(p.head_dim, pl.ncols, g, ks, pl.tiles_per_cta_max);
+    if ((int)lay.total <= kSmemBudget) {
+      pl.k_stages = ks;
+      pl.lay = lay;
+      pl.ok = true;
+      break;
+    }
+  }
+  return pl;
+}
+
+struct FusedWorkspace {
+  size_t partial_off, lse2_off, ctl_off, ctl_bytes, total;
+};
+
+FusedWorkspace fused_workspace(const ScoreProblem& p) {
+  const size_t n_slabs = (size_t)p.n_layers * p.n_kv_heads;
+  FusedWorkspace w;
+  w.partial_off = 0;
+  w.lse2_off = align_up(n_slabs * kFusedMaxCtas * 64 * sizeof(float2), 256);
+  w.ctl_off = align_up(w.lse2_off + n_slabs * 64 * sizeof(float), 256);
+  w.ctl_bytes = align_up(2 * n_slabs * sizeof(unsigned), 256);
+  w.total = w.ctl_off + w.ctl_bytes;
+  return w;
+}
+
+template <int D, int NCOLS, int G>
+int32_t launch_fused(const FusedMaps& maps, const FusedArgs& args, const FusedPlan& pl, cudaStream_t stream) {
+  auto kern = score_fused_kernel<D, NCOLS, G>;
+  const int smem_bytes = (int)pl.lay.total + 1024;
+  SPF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+  kern<<<pl.n_cta, kThreads, smem_bytes, stream>>>(maps, args);
+  SPF_CUDA_CHECK(cudaGetLastError());
+  return SPF_OK;
+}
+
+template <int D, int NCOLS>
+int32_t launch_fused_g(int g, const FusedMaps& maps, const FusedArgs& args, const FusedPlan& pl, cudaStream_t stream) {
+  // a thread owns NCOLS / 2 query rows, which must hold whole GQA groups
+  if constexpr (NCOLS >= 16) {
+    switch (g) {
+      case 1: return launch_fused<D, NCOLS, 1>(maps, args, pl, stream);
+      case 2: return launch_fused<D, NCOLS, 2>(maps, args, pl, stream);
+      case 4: return launch_fused<D, NCOLS, 4>(maps, args, pl, stream);
+      default: return launch_fused<D, NCOLS, 8>(maps, args, pl, stream);
+    }
+  }
+  return SPF_ERR_UNSUPPORTED;
+}
+
+template <int D>
+int32_t launch_fused_n(int ncols, int g, const FusedMaps& maps, const FusedArgs& args, const FusedPlan& pl, cudaStream_t stream) {
+  switch (ncols) {
+    case 16: return launch_fused_g<D, 16>(g, maps, args, pl, stream);
+    case 32: return launch_fused_g<D, 32>(g, maps, args, pl, stream);
+    default: return launch_fused_g<D, 64>(g, maps, args, pl, stream);
+  }
+}
+
+}  // namespace
+
+bool score_fused_supported(const ScoreProblem& p, int sm_count) { return make_plan(p, sm_count).ok; }
+
+size_t score_fused_workspace_bytes(const ScoreProblem& p) { return fused_workspace(p).total; }
+
+int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count, int32_t* dev_status, cudaStream_t stream) {
+  const FusedPlan pl = make_plan(p, sm_count);
+  if (!pl.ok) return fail(SPF_ERR_UNSUPPORTED, "spf_score: shape not covered by the fused path");
+  EncodeTiledFn encode = encode_fn();
+  if (encode == nullptr) return fail(SPF_ERR_CUDA, "spf_score: cuTensorMapEncodeTiled is not available from the driver");
+  const FusedWorkspace w = fused_workspace(p);
+  char* base = static_cast<char*>(workspace);
+
+  FusedMaps maps;
+  const int d = p.head_dim, g = p.group, m = p.n_lookahead;
+  const int n_slabs = p.n_layers * p.n_kv_heads;
+  {
+    const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)g, (cuuint64_t)m, (cuuint64_t)n_slabs};
+    const cuuint64_t strides[3] = {(cuuint64_t)m * d * 2, (cuuint64_t)d * 2, (cuuint64_t)g * m * d * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)g, (cuuint32_t)m, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = encode(&maps.q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(p.q), dims, strides, box,
+                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(SPF_ERR_CUDA, "spf_score: encoding the query tensor map failed (CUresult %d)", (int)r);
+  }
+  for (int l = 0; l < p.n_layers; ++l) {
+    const cuuint64_t head_stride = p.n_kv_heads > 1 ? (cuuint64_t)p.stride_head : (cuuint64_t)p.stride_tok * p.n_tokens;
+    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)p.n_tokens, (cuuint64_t)p.n_kv_heads};
+    const cuuint64_t strides[2] = {(cuuint64_t)p.stride_tok * 2, head_stride * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kTileKeys, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = encode(&maps.k[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(p.k.p[l]), dims, strides,
+                              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+      return fail(SPF_ERR_CUDA, "spf_score: encoding the key tensor map of layer %d failed (CUresult %d)", l, (int)r);
+  }
+
+  FusedArgs args{};
+  for (int l = 0; l < p.n_layers; ++l) args.k_layers[l] = p.k.p[l];
+  args.q = p.q;
+  args.n_tokens = p.n_tokens;
+  args.stride_head = p.stride_head;
+  args.stride_tok = p.stride_tok;
+  args.n_layers = p.n_layers;
+  args.n_kv_heads = p.n_kv_heads;
+  args.n_lookahead = m;
+  args.n_tiles = pl.n_tiles;
+  args.tiles_per_cta_max = pl.tiles_per_cta_max;
+  args.lag = 1;
+  args.k_stages = pl.k_stages;
+  args.c = p.c_log2;
+  args.inv_c = 1.0f / p.c_log2;
+  args.partial = reinterpret_cast<float2*>(base + w.partial_off);
+  args.lse2 = reinterpret_cast<float*>(base + w.lse2_off);
+  args.counters = reinterpret_cast<unsigned*>(base + w.ctl_off);
+  args.ready = args.counters + n_slabs;
+  args.lse_out = p.lse_out;
+  args.importance = p.importance;
+  args.dev_status = dev_status;
+
+  SPF_CUDA_CHECK(cudaMemsetAsync(base + w.ctl_off, 0, w.ctl_bytes, stream));
+  if (d == 64) return launch_fused_n<64>(pl.ncols, g, maps, args, pl, stream);
+  return launch_fused_n<128>(pl.ncols, g, maps, args, pl, stream);
+}
+
+}  // namespace spf

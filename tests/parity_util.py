@@ -17,6 +17,7 @@ def oracle_run(prompt, keep):
 
 
 def gpu_run(prompt, keep, selector=None):
+    """Runs the whole CUDA path; a non-zero device status (timeout, range) fails the test."""
     import paper_2603_02631_b200 as spf
     cfg = prompt.cfg
     dp = prompt.to("cuda")

@@ -11,10 +11,13 @@ from parity_util import (assert_importance_close, assert_selection_matches, comp
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module")
-def spf():
+@pytest.fixture(scope="module", params=["general", "fused"])
+def spf(request):
+    """The package with spf_score pinned to one of its two kernel paths (restored afterwards)."""
     import paper_2603_02631_b200 as mod
-    return mod
+    previous = mod.spf_set_score_path({"general": 1, "fused": 2}[request.param])
+    yield mod
+    mod.spf_set_score_path(previous)
 
 
 def test_tiny_config_end_to_end(spf):

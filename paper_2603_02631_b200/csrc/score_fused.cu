@@ -27,16 +27,20 @@
 // (base-2 units): sums stay finite unless some key beats the samples by more than 2^187, in which
 // case the row's sum becomes inf and SPF_ERR_RANGE is reported.
 //
-// Cross-CTA step.  After visit 1 of a slab every CTA publishes its partial (ref, sum) per row; the
-// CTA that arrives last merges them into lse2[slab][row] and raises a flag that the visit-2 side of
-// every CTA waits for.  Because visit 1 never waits on another CTA and all CTAs are co-resident,
-// the flags always get raised.
+// Cross-CTA step.  All CTAs use the same reference for a row (its logit against one fixed sample key),
+// so their partial sums can simply be added.  To make the total independent of the order in which
+// CTAs arrive, the fp32 partial sums are added EXACTLY: each is split over two 40-bit limbs of a
+// 280-bit fixed-point accumulator per row (64-bit integer atomics, no carries needed), which covers
+// every finite fp32 value.  A counter per slab tells the visit-2 side of every CTA when all shares
+// are in; it then converts the accumulator to lse itself.  Results are bit-identical from run to run.
+// Because visit 1 never waits on another CTA and all CTAs are co-resident, the counters always fill.
 //
 // Every wait in this file is bounded: on expiry the kernel records SPF_ERR_TIMEOUT, drains and
 // returns normally.
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -47,12 +51,13 @@ namespace {
 
 constexpr int kTileKeys = 128;
 constexpr int kThreads = 384;          // warp 0 TMA, 1 MMA, 2 control, 3 idle, 4..11 epilogue
+constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accumulators (covers every finite fp32)
+constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
 constexpr int kEpiWarps = 8;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kQStages = 3;
 constexpr int kTmemStages = 4;
 constexpr int kRefSlots = 8;
-constexpr int kMaxSamples = 4;
 constexpr float kRefMargin = 60.f;     // base-2 units added to the sampled reference logit
 constexpr unsigned long long kTimeoutNs = 2000000000ull;
 constexpr int kSubTileBytes = kTileKeys * 128;  // 128 keys x 64 bf16, one swizzle-128B tile
@@ -69,10 +74,8 @@ struct FusedArgs {
   int64_t n_tokens, stride_head, stride_tok;
   int n_layers, n_kv_heads, n_lookahead, n_tiles, tiles_per_cta_max, lag, k_stages;
   float c, inv_c;
-  float2* partial;        // [slab][cta][NCOLS] (ref, sum)
-  float* lse2;            // [slab][NCOLS]
-  unsigned* counters;     // [slab] arrivals of visit 1
-  unsigned* ready;        // [slab] 1 once lse2[slab] is final
+  unsigned long long* limbs;  // [slab][NCOLS][kLimbStride] exact fixed-point sums of exp2(c*q.k - ref) over all keys
+  unsigned* counters;     // [slab] epilogue warps (8 per CTA) that have added their share of the slab's row sums
   float* lse_out;         // optional [L][Hq][m], natural log
   float* importance;      // [N]
   int32_t* dev_status;    // optional
@@ -140,13 +143,13 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, co
   return __all_sync(0xffffffffu, mbar_wait(bar, parity, ab));
 }
 
-// Waits until *flag (global) becomes non-zero, with acquire semantics.
-__device__ __forceinline__ bool flag_wait(const unsigned* flag, const Abort& ab) {
+// Waits until *counter (global) has reached `target`, with acquire semantics.
+__device__ __forceinline__ bool count_wait(const unsigned* counter, unsigned target, const Abort& ab) {
   unsigned long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
     unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-    if (v != 0u) return true;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= target) return true;
     if ((it & 15u) == 15u) {
       if (*ab.flag) return false;
       const unsigned long long now = global_timer();
@@ -283,7 +286,7 @@ __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, i
   s.offs_off = o;     o += kQSubTileBytes;
   s.amax_off = o;     o += (uint32_t)tiles_per_cta_max * (ncols / group) * kTileKeys * 4;
   s.ref_off = o;      o += kRefSlots * 64 * 4;
-  s.red_off = o;      o += 4 * 64 * 4;
+  s.red_off = o;      o += 2 * 4 * 64 * 4;
   s.merge_off = o;    o += kEpiThreads * 8;
   s.bar_off = o;      o += 64 * 8;
   s.misc_off = o;     o += 64;
@@ -352,8 +355,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   unsigned char* offs_tile = smem + lay.offs_off;
   float* amax = reinterpret_cast<float*>(smem + lay.amax_off);       // [local tile][NI][128]
   float* ref_slots = reinterpret_cast<float*>(smem + lay.ref_off);   // [kRefSlots][64]
-  float* red = reinterpret_cast<float*>(smem + lay.red_off);         // [4 quadrants][64]
-  float2* merge_buf = reinterpret_cast<float2*>(smem + lay.merge_off);
+  float* red = reinterpret_cast<float*>(smem + lay.red_off);         // [2 buffers][4 quadrants][64]
   volatile int* misc = reinterpret_cast<volatile int*>(smem + lay.misc_off);  // [0] abort, [1] tmem base, [2] is_last
   const Bars bars{smem_u32(smem + lay.bar_off), a.k_stages};
   const Abort ab{misc, a.dev_status};
@@ -492,56 +494,75 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   } else if (warp == 2) {
     // ===== control warp: per-row offsets for the extra MMA step; lane handles rows lane and lane + 32 =====
     bool ok = true;
-    const int n_samples = min(my_tiles, kMaxSamples);
+    const int64_t sample_key = a.n_tokens / 2;                  // the same key for every CTA: one reference per row
     for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
       for (int visit = 0; ok && visit < 2; ++visit) {
         const int slab = visit == 0 ? t : t - a.lag;
         if (slab < 0 || slab >= n_slabs) continue;
         const int x = visit * 2 + (slab & 1);
         const int use = slab >> 1;                              // how often step x was written before
-        if (use > 0) {
-          if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
-        }
         float value[2] = {0.f, 0.f};                            // offsets of rows lane, lane + 32 in q.k units
         if (visit == 0) {
-          // reference logit: max over a few sample keys of this CTA's range, plus a margin
+          // reference logit of a row: its logit against one sample key of the slab, plus a margin
           const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
-          const __nv_bfloat16* kslab = a.k_layers[layer] + hk * a.stride_head;
-          float best[2] = {-INFINITY, -INFINITY};
-          for (int sidx = 0; sidx < n_samples; ++sidx) {
-            const int64_t key = (int64_t)(cta + sidx * n_cta) * kTileKeys;
-            const uint4* krow = reinterpret_cast<const uint4*>(kslab + key * a.stride_tok);
-            float dot[2] = {0.f, 0.f};
-            for (int ch = 0; ch < D / 8; ++ch) {
-              const uint4 kv = __ldg(krow + ch);
-              const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv);
+          const uint4* krow = reinterpret_cast<const uint4*>(a.k_layers[layer] + hk * a.stride_head + sample_key * a.stride_tok);
+          const uint4* qrow[2];
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            const int row = min(lane + 32 * r, rows_real - 1);
+            qrow[r] = reinterpret_cast<const uint4*>(a.q + (((int64_t)slab * G + row % G) * a.n_lookahead + row / G) * D);
+          }
+          float dot[2] = {0.f, 0.f};
+#pragma unroll
+          for (int half = 0; half < D / 64; ++half) {
+            uint4 kv[8], qv[2][8];
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+              kv[ch] = __ldg(krow + half * 8 + ch);
+              qv[0][ch] = __ldg(qrow[0] + half * 8 + ch);
+              qv[1][ch] = __ldg(qrow[1] + half * 8 + ch);
+            }
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+              const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv[ch]);
 #pragma unroll
               for (int r = 0; r < 2; ++r) {
-                const int row = lane + 32 * r;
-                if (row < rows_real) {
-                  const int i = row / G, g = row % G;
-                  const uint4 qv = __ldg(reinterpret_cast<const uint4*>(
-                                             a.q + (((int64_t)slab * G + g) * a.n_lookahead + i) * D) + ch);
-                  const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv);
+                const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv[r][ch]);
 #pragma unroll
-                  for (int e = 0; e < 4; ++e) {
-                    const float2 kf = __bfloat1622float2(k2[e]), qf = __bfloat1622float2(q2[e]);
-                    dot[r] = fmaf(kf.x, qf.x, fmaf(kf.y, qf.y, dot[r]));
-                  }
+                for (int e = 0; e < 4; ++e) {
+                  const float2 kf = __bfloat1622float2(k2[e]), qf = __bfloat1622float2(q2[e]);
+                  dot[r] = fmaf(kf.x, qf.x, fmaf(kf.y, qf.y, dot[r]));
                 }
               }
             }
-            best[0] = fmaxf(best[0], dot[0]);
-            best[1] = fmaxf(best[1], dot[1]);
           }
 #pragma unroll
           for (int r = 0; r < 2; ++r)
-            if (lane + 32 * r < rows_real) value[r] = -(best[r] + kRefMargin * a.inv_c);
+            if (lane + 32 * r < rows_real) value[r] = -(dot[r] + kRefMargin * a.inv_c);
         } else {
-          if (!(ok = __all_sync(0xffffffffu, flag_wait(a.ready + slab, ab)))) break;
+          // all shares of the slab's row sums are in once 8 warps of every CTA have reported
+          if (!(ok = __all_sync(0xffffffffu, count_wait(a.counters + slab, (unsigned)(kEpiWarps * n_cta), ab)))) break;
 #pragma unroll
-          for (int r = 0; r < 2; ++r)
-            if (lane + 32 * r < rows_real) value[r] = -__ldcg(a.lse2 + (int64_t)slab * NCOLS + lane + 32 * r) * a.inv_c;
+          for (int r = 0; r < 2; ++r) {
+            const int row = lane + 32 * r;
+            if (row < rows_real) {
+              const unsigned long long* acc = a.limbs + ((int64_t)slab * NCOLS + row) * kLimbStride;
+              unsigned long long w[kLimbs];
+#pragma unroll
+              for (int i = 0; i < kLimbs; ++i) w[i] = __ldcg(acc + i);
+              double total = 0.0;                              // sum of limb_i * 2^(40 i - 149), exact to 2^-53
+#pragma unroll
+              for (int i = kLimbs - 1; i >= 0; --i) total += __longlong_as_double((long long)(1023 + 40 * i - 149) << 52) * (double)w[i];
+              const float lse2 = ref_slots[(slab % kRefSlots) * 64 + row] + (float)log2(total);
+              if (!(lse2 > -INFINITY && lse2 < INFINITY) && a.dev_status != nullptr)
+                atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
+              value[r] = -lse2 * a.inv_c;
+              if (cta == 0 && a.lse_out != nullptr) a.lse_out[((int64_t)slab * G + row % G) * a.n_lookahead + row / G] = lse2 * kLn2;
+            }
+          }
+        }
+        if (use > 0) {
+          if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
         }
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
@@ -613,56 +634,25 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
             }
           }
           // the lane now holds the warp total of column hh * CH + lane / (32 / CH)
+          // the lane now holds the warp total of column hh * CH + lane / (32 / CH): add it, exactly, to the
+          // row's fixed-point accumulator (value = mantissa * 2^(p - 149), p = biased exponent - 1)
           constexpr int kLanesPerCol = 32 / CH;
-          if (lane % kLanesPerCol == 0) red[quad * 64 + hh * CH + lane / kLanesPerCol] = sum[0];
-          if (!(ok = es.sync(lane, ab))) break;
-          if (et < NCOLS) {
-            const float total = red[et] + red[64 + et] + red[128 + et] + red[192 + et];
-            const float ref = ref_slots[(slab % kRefSlots) * 64 + et];
-            __stcg(a.partial + ((int64_t)slab * n_cta + cta) * NCOLS + et, make_float2(ref, total));
-            __threadfence();
-          }
-          if (!(ok = es.sync(lane, ab))) break;
-          if (et == 0) {
-            const unsigned old = atomicAdd(a.counters + slab, 1u);
-            misc[2] = old == (unsigned)(n_cta - 1);
-          }
-          if (!(ok = es.sync(lane, ab))) break;
-          if (misc[2]) {
-            // last CTA to finish visit 1 of this slab: merge all partials into lse2[slab][:]
-            __threadfence();
-            constexpr int kSubsets = kEpiThreads / NCOLS;
-            const int col = et % NCOLS, sub = et / NCOLS;
-            float m = -INFINITY, z = 0.f;
-            for (int b = sub; b < n_cta; b += kSubsets) {
-              const float2 p = __ldcg(a.partial + ((int64_t)slab * n_cta + b) * NCOLS + col);
-              const float v = p.x + log2f(p.y);                // log2 of this CTA's share of the row sum
-              const float mm = fmaxf(m, v);
-              z = z * exp2f(m - mm) + exp2f(v - mm);
-              m = mm;
+          if (lane % kLanesPerCol == 0) {
+            const uint32_t bits = __float_as_uint(sum[0]);
+            const uint32_t expo = bits >> 23;                  // sums are non-negative: no sign bit
+            if (expo == 255u) {
+              if (a.dev_status != nullptr) atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
+            } else if (expo != 0u) {
+              const unsigned long long mant = (unsigned long long)((bits & 0x7FFFFFu) | 0x800000u);
+              const uint32_t pos = expo - 1u, limb = pos / 40u, off = pos % 40u;
+              unsigned long long* acc = a.limbs + ((int64_t)slab * NCOLS + hh * CH + lane / kLanesPerCol) * kLimbStride + limb;
+              const unsigned long long lo = (mant << off) & ((1ull << 40) - 1ull), hi = mant >> (40u - off);
+              atomicAdd(acc, lo);
+              if (hi != 0ull) atomicAdd(acc + 1, hi);
             }
-            merge_buf[et] = make_float2(m, z);
-            if (!(ok = es.sync(lane, ab))) break;
-            if (et < NCOLS) {
-              float mm = -INFINITY;
-              for (int s2 = 0; s2 < kSubsets; ++s2) mm = fmaxf(mm, merge_buf[s2 * NCOLS + et].x);
-              float zz = 0.f;
-              for (int s2 = 0; s2 < kSubsets; ++s2) {
-                const float2 p = merge_buf[s2 * NCOLS + et];
-                if (p.x > -INFINITY) zz += p.y * exp2f(p.x - mm);
-              }
-              const float lse2 = mm + log2f(zz);
-              __stcg(a.lse2 + (int64_t)slab * NCOLS + et, lse2);
-              const int i = et / G, g = et % G;
-              if (a.lse_out != nullptr && i < a.n_lookahead)
-                a.lse_out[((int64_t)slab * G + g) * a.n_lookahead + i] = lse2 * kLn2;
-              if (et < rows_real && !(lse2 > -INFINITY && lse2 < INFINITY) && a.dev_status != nullptr)
-                atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
-              __threadfence();
-            }
-            if (!(ok = es.sync(lane, ab))) break;
-            if (et == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.ready + slab), "r"(1u) : "memory");
           }
+          __syncwarp();
+          if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(a.counters + slab), "r"(1u) : "memory");
         } else {
           // ---------------- visit 2: running max over (layer, head) of q.k - lse/c ----------------
           for (int lt = 0; lt < my_tiles; ++lt) {
@@ -767,18 +757,27 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
   return pl;
 }
 
+// How many slabs the second visit runs behind the first.  Two leaves a full slab of time for the
+// cross-CTA merge of the row sums; the environment variable SPF_FUSED_LAG (1..4) overrides it for tuning.
+int fused_lag(int n_slabs) {
+  int lag = 2;
+  if (const char* env = getenv("SPF_FUSED_LAG")) {
+    const int v = atoi(env);
+    if (v >= 1 && v <= 4) lag = v;
+  }
+  return std::max(1, std::min(lag, n_slabs));
+}
+
 struct FusedWorkspace {
-  size_t partial_off, lse2_off, ctl_off, ctl_bytes, total;
+  size_t limbs_off, counters_off, total;   // both are cleared before every launch
 };
 
 FusedWorkspace fused_workspace(const ScoreProblem& p) {
   const size_t n_slabs = (size_t)p.n_layers * p.n_kv_heads;
   FusedWorkspace w;
-  w.partial_off = 0;
-  w.lse2_off = align_up(n_slabs * kFusedMaxCtas * 64 * sizeof(float2), 256);
-  w.ctl_off = align_up(w.lse2_off + n_slabs * 64 * sizeof(float), 256);
-  w.ctl_bytes = align_up(2 * n_slabs * sizeof(unsigned), 256);
-  w.total = w.ctl_off + w.ctl_bytes;
+  w.limbs_off = 0;
+  w.counters_off = align_up(n_slabs * 64 * kLimbStride * sizeof(unsigned long long), 256);
+  w.total = align_up(w.counters_off + n_slabs * sizeof(unsigned), 256);
   return w;
 }
 
@@ -866,19 +865,17 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   args.n_lookahead = m;
   args.n_tiles = pl.n_tiles;
   args.tiles_per_cta_max = pl.tiles_per_cta_max;
-  args.lag = 1;
+  args.lag = fused_lag(n_slabs);
   args.k_stages = pl.k_stages;
   args.c = p.c_log2;
   args.inv_c = 1.0f / p.c_log2;
-  args.partial = reinterpret_cast<float2*>(base + w.partial_off);
-  args.lse2 = reinterpret_cast<float*>(base + w.lse2_off);
-  args.counters = reinterpret_cast<unsigned*>(base + w.ctl_off);
-  args.ready = args.counters + n_slabs;
+  args.limbs = reinterpret_cast<unsigned long long*>(base + w.limbs_off);
+  args.counters = reinterpret_cast<unsigned*>(base + w.counters_off);
   args.lse_out = p.lse_out;
   args.importance = p.importance;
   args.dev_status = dev_status;
 
-  SPF_CUDA_CHECK(cudaMemsetAsync(base + w.ctl_off, 0, w.ctl_bytes, stream));
+  SPF_CUDA_CHECK(cudaMemsetAsync(base, 0, w.total, stream));
   if (d == 64) return launch_fused_n<64>(pl.ncols, g, maps, args, pl, stream);
   return launch_fused_n<128>(pl.ncols, g, maps, args, pl, stream);
 }

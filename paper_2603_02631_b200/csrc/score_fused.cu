@@ -50,7 +50,7 @@ namespace spf {
 namespace {
 
 constexpr int kTileKeys = 128;
-constexpr int kThreads = 384;          // warp 0 TMA, 1 MMA, 2 control, 3 idle, 4..11 epilogue
+constexpr int kThreads = 384;          // warp 0 TMA, 1 MMA, 2 control, 3 publisher, 4..11 epilogue
 constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accumulators (covers every finite fp32)
 constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
 constexpr int kEpiWarps = 8;
@@ -58,6 +58,7 @@ constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kQStages = 3;
 constexpr int kTmemStages = 4;
 constexpr int kRefSlots = 8;
+constexpr int kPubSlots = 4;
 constexpr float kRefMargin = 60.f;     // base-2 units added to the sampled reference logit
 constexpr unsigned long long kTimeoutNs = 2000000000ull;
 constexpr int kSubTileBytes = kTileKeys * 128;  // 128 keys x 64 bf16, one swizzle-128B tile
@@ -75,7 +76,7 @@ struct FusedArgs {
   int n_layers, n_kv_heads, n_lookahead, n_tiles, tiles_per_cta_max, lag, k_stages;
   float c, inv_c;
   unsigned long long* limbs;  // [slab][NCOLS][kLimbStride] exact fixed-point sums of exp2(c*q.k - ref) over all keys
-  unsigned* counters;     // [slab] epilogue warps (8 per CTA) that have added their share of the slab's row sums
+  unsigned* counters;     // [slab] CTAs whose share of the slab's row sums is in the accumulators
   float* lse_out;         // optional [L][Hq][m], natural log
   float* importance;      // [N]
   int32_t* dev_status;    // optional
@@ -177,6 +178,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// True in exactly one lane of the (converged) warp, the same lane every time.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
+  return pred != 0;
+}
+
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -207,34 +215,45 @@ __host__ __device__ constexpr uint32_t instr_desc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileKeys >> 4) << 24);
 }
 
+// TMEM -> registers, split in two so that a load can be in flight while the previous tile is processed:
+// tmem_issue starts the (asynchronous) load of N consecutive columns of the warp's 32 lanes, tmem_wait
+// completes it.  The registers are listed as in/out operands of the wait so that no use can move above it.
 template <int N>
-__device__ __forceinline__ void tmem_load(uint32_t taddr, float (&v)[N]);
+__device__ __forceinline__ void tmem_issue(uint32_t taddr, uint32_t (&r)[N]);
+template <int N>
+__device__ __forceinline__ void tmem_wait(uint32_t (&r)[N]);
 
 template <>
-__device__ __forceinline__ void tmem_load<8>(uint32_t taddr, float (&v)[8]) {
-  uint32_t r[8];
+__device__ __forceinline__ void tmem_issue<8>(uint32_t taddr, uint32_t (&r)[8]) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 template <>
-__device__ __forceinline__ void tmem_load<16>(uint32_t taddr, float (&v)[16]) {
-  uint32_t r[16];
+__device__ __forceinline__ void tmem_wait<8>(uint32_t (&r)[8]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
+               :
+               : "memory");
+}
+template <>
+__device__ __forceinline__ void tmem_issue<16>(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 template <>
-__device__ __forceinline__ void tmem_load<32>(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+__device__ __forceinline__ void tmem_wait<16>(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :
+               : "memory");
+}
+template <>
+__device__ __forceinline__ void tmem_issue<32>(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,"
       "%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
@@ -243,9 +262,16 @@ __device__ __forceinline__ void tmem_load<32>(uint32_t taddr, float (&v)[32]) {
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+template <>
+__device__ __forceinline__ void tmem_wait<32>(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                 "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                 "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
 }
 
 // Byte offset of element (row, col) of a [rows x 64] bf16 tile stored with the 128-byte swizzle.
@@ -308,8 +334,9 @@ struct Bars {
   __device__ uint32_t o_free(int x) const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 4 + x); }
   __device__ uint32_t epi_sync() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 8); }
   __device__ uint32_t mma_done() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 9); }
+  __device__ uint32_t pub_ready(int b) const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 10 + b); }
 };
-// 2 * 8 + 2 * 3 + 2 * 4 + 10 = 40 barriers at most; the block has room for 64.
+// 2 * 8 + 2 * 3 + 2 * 4 + 14 = 44 barriers at most; the block has room for 64.
 
 struct Ring {
   int stage = 0;
@@ -389,6 +416,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     }
     mbar_init(bars.epi_sync(), kEpiWarps);
     mbar_init(bars.mma_done(), 1);
+    for (int b = 0; b < kPubSlots; ++b) mbar_init(bars.pub_ready(b), kEpiWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // zero the query stages (rows the TMA box does not cover must read as zero), the offsets tile and the
@@ -447,48 +475,60 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       }
     }
   } else if (warp == 1) {
-    // ===== MMA issuer =====
-    if (lane == 0) {
+    // ===== MMA issuer: the whole warp walks the loop (so addresses and descriptors stay warp-uniform),
+    // one elected lane issues the tensor-core instructions =====
+    {
       Ring kr(a.k_stages), qr(kQStages), tr(kTmemStages);
       constexpr uint32_t idesc = instr_desc(NCOLS);
       const uint64_t ones_desc = smem_desc(smem_u32(ones_tile));
       const uint64_t offs_desc = smem_desc(smem_u32(offs_tile));
+      const uint64_t k_desc0 = smem_desc(smem_u32(k_tiles));
+      const uint64_t q_desc0 = smem_desc(smem_u32(q_tiles));
       bool ok = true;
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
         for (int visit = 0; ok && visit < 2; ++visit) {
           const int slab = visit == 0 ? t : t - a.lag;
           if (slab < 0 || slab >= n_slabs) continue;
           const int x = visit * 2 + (slab & 1);                 // which 16-wide step of the offsets tile
-          if (!(ok = mbar_wait(bars.q_full(qr.stage), qr.phase, ab))) break;
-          if (!(ok = mbar_wait(bars.o_ready(x), (uint32_t)(slab >> 1) & 1u, ab))) break;
+          if (!(ok = mbar_wait_warp(bars.q_full(qr.stage), qr.phase, ab))) break;
+          if (!(ok = mbar_wait_warp(bars.o_ready(x), (uint32_t)(slab >> 1) & 1u, ab))) break;
+          const uint64_t bd0 = q_desc0 + (uint64_t)((qr.stage * KSUB * kQSubTileBytes) >> 4);
           for (int lt = 0; lt < my_tiles; ++lt) {
-            if (!(ok = mbar_wait(bars.k_full(kr.stage), kr.phase, ab))) break;
-            if (!(ok = mbar_wait(bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
+            if (!(ok = mbar_wait_warp(bars.k_full(kr.stage), kr.phase, ab))) break;
+            if (!(ok = mbar_wait_warp(bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(tr.stage * NCOLS);
+            const uint64_t ad0 = k_desc0 + (uint64_t)((kr.stage * KSUB * kSubTileBytes) >> 4);
+            if (elect_one()) {
 #pragma unroll
-            for (int h = 0; h < KSUB; ++h) {
-              const uint64_t ad = smem_desc(smem_u32(k_tiles + (kr.stage * KSUB + h) * kSubTileBytes));
-              const uint64_t bd = smem_desc(smem_u32(q_tiles + (qr.stage * KSUB + h) * kQSubTileBytes));
+              for (int h = 0; h < KSUB; ++h) {
 #pragma unroll
-              for (int ks = 0; ks < 4; ++ks) tc_mma(d_tmem, ad + 2u * ks, bd + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
+                for (int ks = 0; ks < 4; ++ks)
+                  tc_mma(d_tmem, ad0 + (uint64_t)((h * kSubTileBytes) >> 4) + 2u * ks,
+                         bd0 + (uint64_t)((h * kQSubTileBytes) >> 4) + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
+              }
+              tc_mma(d_tmem, ones_desc + 2u * x, offs_desc + 2u * x, idesc, 1u);
+              tc_commit(bars.k_empty(kr.stage));
+              tc_commit(bars.t_full(tr.stage));
             }
-            tc_mma(d_tmem, ones_desc + 2u * x, offs_desc + 2u * x, idesc, 1u);
-            tc_commit(bars.k_empty(kr.stage));
-            tc_commit(bars.t_full(tr.stage));
+            __syncwarp();
             kr.advance();
             tr.advance();
           }
           if (!ok) break;
-          tc_commit(bars.q_empty(qr.stage));
-          tc_commit(bars.o_free(x));
+          if (elect_one()) {
+            tc_commit(bars.q_empty(qr.stage));
+            tc_commit(bars.o_free(x));
+          }
+          __syncwarp();
           qr.advance();
         }
       }
       // leave only after everything issued has completed and signalled its barriers
       if (ok) {
-        tc_commit(bars.mma_done());
-        mbar_wait(bars.mma_done(), 0u, ab);
+        if (elect_one()) tc_commit(bars.mma_done());
+        __syncwarp();
+        mbar_wait_warp(bars.mma_done(), 0u, ab);
       }
     }
   } else if (warp == 2) {
@@ -540,8 +580,8 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
           for (int r = 0; r < 2; ++r)
             if (lane + 32 * r < rows_real) value[r] = -(dot[r] + kRefMargin * a.inv_c);
         } else {
-          // all shares of the slab's row sums are in once 8 warps of every CTA have reported
-          if (!(ok = __all_sync(0xffffffffu, count_wait(a.counters + slab, (unsigned)(kEpiWarps * n_cta), ab)))) break;
+          // all shares of the slab's row sums are in once every CTA has reported
+          if (!(ok = __all_sync(0xffffffffu, count_wait(a.counters + slab, (unsigned)n_cta, ab)))) break;
 #pragma unroll
           for (int r = 0; r < 2; ++r) {
             const int row = lane + 32 * r;
@@ -577,6 +617,16 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         if (lane == 0) mbar_arrive(bars.o_ready(x));
       }
     }
+  } else if (warp == 3) {
+    // ===== publisher: once the eight epilogue warps have added their shares of a slab's row sums, order those
+    // additions before the arrival count and report this CTA (keeps the fence off the epilogue warps) =====
+    if (lane == 0) {
+      for (int slab = 0; slab < n_slabs; ++slab) {
+        if (!mbar_wait(bars.pub_ready(slab % kPubSlots), (uint32_t)(slab / kPubSlots) & 1u, ab)) break;
+        __threadfence();
+        atomicAdd(a.counters + slab, 1u);
+      }
+    }
   } else if (warp >= 4) {
     // ===== epilogue: 8 warps; warp % 4 picks the TMEM lane quadrant (keys), warps 4-7 / 8-11 the column half =====
     const int quad = warp & 3;
@@ -590,27 +640,57 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       for (int visit = 0; ok && visit < 2; ++visit) {
         const int slab = visit == 0 ? t : t - a.lag;
         if (slab < 0 || slab >= n_slabs) continue;
-        if (visit == 0) {
-          // ---------------- visit 1: per-thread sums of exp2 over the thread's keys ----------------
-          float sum[CH];
+        // tile loop shared by both visits: the TMEM load of tile lt + 1 is in flight while tile lt is processed
+        float sum[CH];
 #pragma unroll
-          for (int j = 0; j < CH; ++j) sum[j] = 0.f;
-          for (int lt = 0; lt < my_tiles; ++lt) {
-            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
-            tc_fence_after();
-            float v[CH];
-            tmem_load<CH>(tmem_base + lane_addr + (uint32_t)(tr.stage * NCOLS + hh * CH), v);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
-            tr.advance();
+        for (int j = 0; j < CH; ++j) sum[j] = 0.f;
+        auto process = [&](const uint32_t (&r)[CH], int lt) {
+          if (visit == 0) {
+            // visit 1: per-thread sums of exp2 over the thread's keys
             const int64_t key = (int64_t)(cta + lt * n_cta) * kTileKeys + quad * 32 + lane;
             if (key < a.n_tokens) {
 #pragma unroll
-              for (int j = 0; j < CH; ++j) sum[j] += fast_exp2(v[j] * a.c);
+              for (int j = 0; j < CH; ++j) sum[j] += fast_exp2(__uint_as_float(r[j]) * a.c);
+            }
+          } else {
+            // visit 2: running max over (layer, head) of q.k - lse/c
+            float* slot = amax + ((int64_t)lt * NI + hh * (CH / G)) * kTileKeys + quad * 32 + lane;
+#pragma unroll
+            for (int ii = 0; ii < CH / G; ++ii) {
+              float mx = __uint_as_float(r[ii * G]);
+#pragma unroll
+              for (int g = 1; g < G; ++g) mx = fmaxf(mx, __uint_as_float(r[ii * G + g]));
+              if (hh * (CH / G) + ii < a.n_lookahead) slot[ii * kTileKeys] = fmaxf(slot[ii * kTileKeys], mx);
             }
           }
-          if (!ok) break;
+        };
+        auto start_load = [&](uint32_t (&r)[CH]) -> bool {
+          if (!mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab)) return false;
+          tc_fence_after();
+          tmem_issue<CH>(tmem_base + lane_addr + (uint32_t)(tr.stage * NCOLS + hh * CH), r);
+          return true;
+        };
+        auto finish_load = [&](uint32_t (&r)[CH]) {
+          tmem_wait<CH>(r);
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));   // the stage can be overwritten: its data is in registers
+          tr.advance();
+        };
+        uint32_t ra[CH], rb[CH];
+        if (!(ok = start_load(ra))) break;
+        for (int lt = 0; lt < my_tiles; lt += 2) {
+          finish_load(ra);
+          if (lt + 1 < my_tiles && !(ok = start_load(rb))) break;
+          process(ra, lt);
+          if (lt + 1 < my_tiles) {
+            finish_load(rb);
+            if (lt + 2 < my_tiles && !(ok = start_load(ra))) break;
+            process(rb, lt + 1);
+          }
+        }
+        if (!ok) break;
+        if (visit == 0) {
           // reduce over the 32 keys of the warp: transposing butterfly while more than one column is
           // left per thread, plain butterfly afterwards
           {
@@ -633,7 +713,6 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
               }
             }
           }
-          // the lane now holds the warp total of column hh * CH + lane / (32 / CH)
           // the lane now holds the warp total of column hh * CH + lane / (32 / CH): add it, exactly, to the
           // row's fixed-point accumulator (value = mantissa * 2^(p - 149), p = biased exponent - 1)
           constexpr int kLanesPerCol = 32 / CH;
@@ -651,28 +730,9 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
               if (hi != 0ull) atomicAdd(acc + 1, hi);
             }
           }
+          // hand over to the publisher warp, which makes the additions visible and counts this CTA in
           __syncwarp();
-          if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(a.counters + slab), "r"(1u) : "memory");
-        } else {
-          // ---------------- visit 2: running max over (layer, head) of q.k - lse/c ----------------
-          for (int lt = 0; lt < my_tiles; ++lt) {
-            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
-            tc_fence_after();
-            float v[CH];
-            tmem_load<CH>(tmem_base + lane_addr + (uint32_t)(tr.stage * NCOLS + hh * CH), v);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
-            tr.advance();
-            float* slot = amax + ((int64_t)lt * NI + hh * (CH / G)) * kTileKeys + quad * 32 + lane;
-#pragma unroll
-            for (int ii = 0; ii < CH / G; ++ii) {
-              float mx = v[ii * G];
-#pragma unroll
-              for (int g = 1; g < G; ++g) mx = fmaxf(mx, v[ii * G + g]);
-              if (hh * (CH / G) + ii < a.n_lookahead) slot[ii * kTileKeys] = fmaxf(slot[ii * kTileKeys], mx);
-            }
-          }
+          if (lane == 0) mbar_arrive(bars.pub_ready(slab % kPubSlots));
         }
       }
     }

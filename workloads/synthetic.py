@@ -91,6 +91,9 @@ CONFIGS = {
     # Long context: the configuration the headline metric is quoted on.
     "long128k": WorkloadConfig("long128k", 16, 32, 8, 64, 16, (131072,), 32, (0.10,), rank=16,
                                n_needles=256, n_strong=64, needle_len=(16, 128), recency=True, seed=3),
+    # The long-context geometry cut to 4 layers (K cache 512 MiB): sized for profiler captures.
+    "long128k_l4": WorkloadConfig("long128k_l4", 4, 32, 8, 64, 16, (131072,), 32, (0.10,), rank=16,
+                                  n_needles=256, n_strong=64, needle_len=(16, 128), recency=True, seed=3),
     # Ragged batch of 8 prompts.
     "ragged8": WorkloadConfig("ragged8", 28, 16, 8, 128, 8, _ragged_lengths(4, 8, 16384, 131072), 32,
                               (0.10,), rank=16, n_needles=64, n_strong=16, needle_len=(16, 128),

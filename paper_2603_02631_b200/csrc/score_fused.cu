@@ -19,13 +19,10 @@
 // and sees all query rows of it: the max over heads is in-thread, and the sum over keys is kept
 // per thread and reduced across threads only once per slab.
 //
-// Folded offsets.  An extra 16-wide MMA step multiplies a constant tile of ones (key side) with a
-// small tile holding, per query row, an offset split into three bf16 terms.  Visit 1 uses
-// -ref/c (a reference logit, so that exp2 cannot overflow), visit 2 uses -lse/c.  The subtraction
-// thus happens in the tensor core's fp32 accumulator and costs no ALU instruction per logit.
-// The reference of a row is the largest logit among a few sample keys of the CTA plus a margin of 60
-// (base-2 units): sums stay finite unless some key beats the samples by more than 2^187, in which
-// case the row's sum becomes inf and SPF_ERR_RANGE is reported.
+// Row offsets.  Visit 1 subtracts a per-row reference ref (in base-2 units) inside the exp2 argument so that
+// exp2 cannot overflow: the reference of a row is its logit against one fixed sample key plus a margin of 60,
+// so sums stay finite unless some key beats the sample by more than 2^187 (then the row's sum becomes inf and
+// SPF_ERR_RANGE is reported).  Visit 2 subtracts lse/c.  A control warp prepares both per slab in shared memory.
 //
 // Cross-CTA step.  All CTAs use the same reference for a row (its logit against one fixed sample key),
 // so their partial sums can simply be added.  To make the total independent of the order in which
@@ -50,7 +47,8 @@ namespace spf {
 namespace {
 
 constexpr int kTileKeys = 128;
-constexpr int kThreads = 384;          // warp 0 TMA, 1 MMA, 2 control, 3 publisher, 4..11 epilogue
+constexpr int kThreads = 384;          // warp 0 TMA, 1 MMA issue, 2 control, 3 publisher, 4..11 epilogue
+constexpr int kIssuers = 1;            // MMA-issuing warps: local tile lt belongs to issuer lt % kIssuers
 constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accumulators (covers every finite fp32)
 constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
 constexpr int kEpiWarps = 8;
@@ -274,33 +272,9 @@ __device__ __forceinline__ void tmem_wait<32>(uint32_t (&r)[32]) {
                : "memory");
 }
 
-// Byte offset of element (row, col) of a [rows x 64] bf16 tile stored with the 128-byte swizzle.
-__device__ __forceinline__ uint32_t swz128(int row, int col) {
-  const int byte = col * 2;
-  return (uint32_t)(row * 128 + ((((byte >> 4) ^ (row & 7)) << 4) | (byte & 15)));
-}
-
-__device__ __forceinline__ unsigned short bf16_bits_rn(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
-__device__ __forceinline__ float bf16_value(unsigned short b) { return __uint_as_float((uint32_t)b << 16); }
-
-// Writes value v (split into three bf16 terms) into row `row`, step `step` of the offsets tile and
-// returns the sum of the three terms, i.e. the offset the tensor core will add.
-__device__ __forceinline__ float write_offset(unsigned char* tile, int row, int step, float v) {
-  const unsigned short t0 = bf16_bits_rn(v);
-  const float r1 = v - bf16_value(t0);
-  const unsigned short t1 = bf16_bits_rn(r1);
-  const float r2 = r1 - bf16_value(t1);
-  const unsigned short t2 = bf16_bits_rn(r2);
-  unsigned short* dst = reinterpret_cast<unsigned short*>(tile + swz128(row, step * 16));
-  dst[0] = t0;
-  dst[1] = t1;
-  dst[2] = t2;
-  return bf16_value(t0) + bf16_value(t1) + bf16_value(t2);
-}
-
 // ---------------------------------------------------------------------------------------------- layout
 struct SmemLayout {
-  uint32_t k_off, q_off, ones_off, offs_off, amax_off, ref_off, red_off, merge_off, bar_off, misc_off, total;
+  uint32_t k_off, q_off, amax_off, ref_off, rowoff_off, bar_off, misc_off, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, int k_stages, int tiles_per_cta_max) {
@@ -308,12 +282,9 @@ __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, i
   uint32_t o = 0;
   s.k_off = o;        o += (uint32_t)k_stages * (d / 64) * kSubTileBytes;
   s.q_off = o;        o += (uint32_t)kQStages * (d / 64) * kQSubTileBytes;
-  s.ones_off = o;     o += kSubTileBytes;
-  s.offs_off = o;     o += kQSubTileBytes;
   s.amax_off = o;     o += (uint32_t)tiles_per_cta_max * (ncols / group) * kTileKeys * 4;
   s.ref_off = o;      o += kRefSlots * 64 * 4;
-  s.red_off = o;      o += 2 * 4 * 64 * 4;
-  s.merge_off = o;    o += kEpiThreads * 8;
+  s.rowoff_off = o;   o += 4 * 64 * 4;
   s.bar_off = o;      o += 64 * 8;
   s.misc_off = o;     o += 64;
   s.total = o;
@@ -336,7 +307,7 @@ struct Bars {
   __device__ uint32_t mma_done() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 9); }
   __device__ uint32_t pub_ready(int b) const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 10 + b); }
 };
-// 2 * 8 + 2 * 3 + 2 * 4 + 14 = 44 barriers at most; the block has room for 64.
+// 2 * 10 + 2 * 3 + 2 * 4 + 14 = 48 barriers at most; the block has room for 64.
 
 struct Ring {
   int stage = 0;
@@ -378,11 +349,9 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   const SmemLayout lay = smem_layout(D, NCOLS, G, a.k_stages, a.tiles_per_cta_max);
   unsigned char* k_tiles = smem + lay.k_off;
   unsigned char* q_tiles = smem + lay.q_off;
-  unsigned char* ones_tile = smem + lay.ones_off;
-  unsigned char* offs_tile = smem + lay.offs_off;
   float* amax = reinterpret_cast<float*>(smem + lay.amax_off);       // [local tile][NI][128]
   float* ref_slots = reinterpret_cast<float*>(smem + lay.ref_off);   // [kRefSlots][64]
-  float* red = reinterpret_cast<float*>(smem + lay.red_off);         // [2 buffers][4 quadrants][64]
+  float* rowoff = reinterpret_cast<float*>(smem + lay.rowoff_off);   // [4 slots][64]: what the epilogue subtracts per row
   volatile int* misc = reinterpret_cast<volatile int*>(smem + lay.misc_off);  // [0] abort, [1] tmem base, [2] is_last
   const Bars bars{smem_u32(smem + lay.bar_off), a.k_stages};
   const Abort ab{misc, a.dev_status};
@@ -404,7 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     }
     for (int s = 0; s < kQStages; ++s) {
       mbar_init(bars.q_full(s), 1);
-      mbar_init(bars.q_empty(s), 1);
+      mbar_init(bars.q_empty(s), kIssuers);
     }
     for (int s = 0; s < kTmemStages; ++s) {
       mbar_init(bars.t_full(s), 1);
@@ -412,26 +381,16 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     }
     for (int x = 0; x < 4; ++x) {
       mbar_init(bars.o_ready(x), 1);
-      mbar_init(bars.o_free(x), 1);
+      mbar_init(bars.o_free(x), kEpiWarps);
     }
     mbar_init(bars.epi_sync(), kEpiWarps);
-    mbar_init(bars.mma_done(), 1);
+    mbar_init(bars.mma_done(), kIssuers);
     for (int b = 0; b < kPubSlots; ++b) mbar_init(bars.pub_ready(b), kEpiWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // zero the query stages (rows the TMA box does not cover must read as zero), the offsets tile and the
-  // constant tile; the constant tile then gets ones in the first three columns of each 16-wide step
+  // zero the query stages: rows the TMA box does not cover must read as zero
   for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kQStages * KSUB * kQSubTileBytes; i += kThreads * 16)
     *reinterpret_cast<uint4*>(q_tiles + i) = make_uint4(0, 0, 0, 0);
-  for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kQSubTileBytes; i += kThreads * 16)
-    *reinterpret_cast<uint4*>(offs_tile + i) = make_uint4(0, 0, 0, 0);
-  for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kSubTileBytes; i += kThreads * 16)
-    *reinterpret_cast<uint4*>(ones_tile + i) = make_uint4(0, 0, 0, 0);
-  __syncthreads();
-  for (int i = threadIdx.x; i < kTileKeys * 4 * 3; i += kThreads) {
-    const int row = i / 12, step = (i % 12) / 3, t = i % 3;
-    *reinterpret_cast<unsigned short*>(ones_tile + swz128(row, step * 16 + t)) = 0x3F80;  // bf16 1.0
-  }
   for (int i = threadIdx.x; i < my_tiles * NI * kTileKeys; i += kThreads) amax[i] = -INFINITY;
   fence_async_smem();
   if (warp == 0) {
@@ -475,13 +434,12 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       }
     }
   } else if (warp == 1) {
-    // ===== MMA issuer: the whole warp walks the loop (so addresses and descriptors stay warp-uniform),
-    // one elected lane issues the tensor-core instructions =====
+    // ===== MMA issuer.  The whole warp walks the loop (addresses and descriptors stay warp-uniform); one elected
+    // lane issues the tensor-core instructions =====
     {
+      const int me = 0;
       Ring kr(a.k_stages), qr(kQStages), tr(kTmemStages);
       constexpr uint32_t idesc = instr_desc(NCOLS);
-      const uint64_t ones_desc = smem_desc(smem_u32(ones_tile));
-      const uint64_t offs_desc = smem_desc(smem_u32(offs_tile));
       const uint64_t k_desc0 = smem_desc(smem_u32(k_tiles));
       const uint64_t q_desc0 = smem_desc(smem_u32(q_tiles));
       bool ok = true;
@@ -489,37 +447,33 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         for (int visit = 0; ok && visit < 2; ++visit) {
           const int slab = visit == 0 ? t : t - a.lag;
           if (slab < 0 || slab >= n_slabs) continue;
-          const int x = visit * 2 + (slab & 1);                 // which 16-wide step of the offsets tile
           if (!(ok = mbar_wait_warp(bars.q_full(qr.stage), qr.phase, ab))) break;
-          if (!(ok = mbar_wait_warp(bars.o_ready(x), (uint32_t)(slab >> 1) & 1u, ab))) break;
           const uint64_t bd0 = q_desc0 + (uint64_t)((qr.stage * KSUB * kQSubTileBytes) >> 4);
           for (int lt = 0; lt < my_tiles; ++lt) {
-            if (!(ok = mbar_wait_warp(bars.k_full(kr.stage), kr.phase, ab))) break;
-            if (!(ok = mbar_wait_warp(bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(tr.stage * NCOLS);
-            const uint64_t ad0 = k_desc0 + (uint64_t)((kr.stage * KSUB * kSubTileBytes) >> 4);
-            if (elect_one()) {
+            if (lt % kIssuers == me) {
+              if (!(ok = mbar_wait_warp(bars.k_full(kr.stage), kr.phase, ab))) break;
+              if (!(ok = mbar_wait_warp(bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
+              tc_fence_after();
+              const uint32_t d_tmem = tmem_base + (uint32_t)(tr.stage * NCOLS);
+              const uint64_t ad0 = k_desc0 + (uint64_t)((kr.stage * KSUB * kSubTileBytes) >> 4);
+              if (elect_one()) {
 #pragma unroll
-              for (int h = 0; h < KSUB; ++h) {
+                for (int h = 0; h < KSUB; ++h) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                  tc_mma(d_tmem, ad0 + (uint64_t)((h * kSubTileBytes) >> 4) + 2u * ks,
-                         bd0 + (uint64_t)((h * kQSubTileBytes) >> 4) + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
+                  for (int ks = 0; ks < 4; ++ks)
+                    tc_mma(d_tmem, ad0 + (uint64_t)((h * kSubTileBytes) >> 4) + 2u * ks,
+                           bd0 + (uint64_t)((h * kQSubTileBytes) >> 4) + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
+                }
+                tc_commit(bars.k_empty(kr.stage));
+                tc_commit(bars.t_full(tr.stage));
               }
-              tc_mma(d_tmem, ones_desc + 2u * x, offs_desc + 2u * x, idesc, 1u);
-              tc_commit(bars.k_empty(kr.stage));
-              tc_commit(bars.t_full(tr.stage));
+              __syncwarp();
             }
-            __syncwarp();
             kr.advance();
             tr.advance();
           }
           if (!ok) break;
-          if (elect_one()) {
-            tc_commit(bars.q_empty(qr.stage));
-            tc_commit(bars.o_free(x));
-          }
+          if (elect_one()) tc_commit(bars.q_empty(qr.stage));   // arrives once this warp's MMAs of the run are done
           __syncwarp();
           qr.advance();
         }
@@ -531,8 +485,18 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         mbar_wait_warp(bars.mma_done(), 0u, ab);
       }
     }
+  } else if (warp == 3) {
+    // ===== publisher: once the eight epilogue warps have added their shares of a slab's row sums, order those
+    // additions before the arrival count and report this CTA (keeps the fence off the epilogue warps) =====
+    if (lane == 0) {
+      for (int slab = 0; slab < n_slabs; ++slab) {
+        if (!mbar_wait(bars.pub_ready(slab % kPubSlots), (uint32_t)(slab / kPubSlots) & 1u, ab)) break;
+        __threadfence();
+        atomicAdd(a.counters + slab, 1u);
+      }
+    }
   } else if (warp == 2) {
-    // ===== control warp: per-row offsets for the extra MMA step; lane handles rows lane and lane + 32 =====
+    // ===== control warp: the per-row offsets the epilogue subtracts; lane handles rows lane and lane + 32 =====
     bool ok = true;
     const int64_t sample_key = a.n_tokens / 2;                  // the same key for every CTA: one reference per row
     for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
@@ -541,7 +505,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         if (slab < 0 || slab >= n_slabs) continue;
         const int x = visit * 2 + (slab & 1);
         const int use = slab >> 1;                              // how often step x was written before
-        float value[2] = {0.f, 0.f};                            // offsets of rows lane, lane + 32 in q.k units
+        float value[2] = {0.f, 0.f};                            // offsets of rows lane, lane + 32
         if (visit == 0) {
           // reference logit of a row: its logit against one sample key of the slab, plus a margin
           const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
@@ -578,7 +542,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
           }
 #pragma unroll
           for (int r = 0; r < 2; ++r)
-            if (lane + 32 * r < rows_real) value[r] = -(dot[r] + kRefMargin * a.inv_c);
+            if (lane + 32 * r < rows_real) value[r] = fmaf(dot[r], a.c, kRefMargin);   // reference, base-2 units
         } else {
           // all shares of the slab's row sums are in once every CTA has reported
           if (!(ok = __all_sync(0xffffffffu, count_wait(a.counters + slab, (unsigned)n_cta, ab)))) break;
@@ -596,7 +560,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
               const float lse2 = ref_slots[(slab % kRefSlots) * 64 + row] + (float)log2(total);
               if (!(lse2 > -INFINITY && lse2 < INFINITY) && a.dev_status != nullptr)
                 atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
-              value[r] = -lse2 * a.inv_c;
+              value[r] = lse2 * a.inv_c;                          // lse in q.k units
               if (cta == 0 && a.lse_out != nullptr) a.lse_out[((int64_t)slab * G + row % G) * a.n_lookahead + row / G] = lse2 * kLn2;
             }
           }
@@ -608,23 +572,12 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         for (int r = 0; r < 2; ++r) {
           const int row = lane + 32 * r;
           if (row < NCOLS) {
-            const float seen = write_offset(offs_tile, row, x, value[r]);
-            if (visit == 0) ref_slots[(slab % kRefSlots) * 64 + row] = -seen * a.c;   // reference in base-2 units
+            rowoff[x * 64 + row] = value[r];
+            if (visit == 0) ref_slots[(slab % kRefSlots) * 64 + row] = value[r];
           }
         }
-        fence_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(bars.o_ready(x));
-      }
-    }
-  } else if (warp == 3) {
-    // ===== publisher: once the eight epilogue warps have added their shares of a slab's row sums, order those
-    // additions before the arrival count and report this CTA (keeps the fence off the epilogue warps) =====
-    if (lane == 0) {
-      for (int slab = 0; slab < n_slabs; ++slab) {
-        if (!mbar_wait(bars.pub_ready(slab % kPubSlots), (uint32_t)(slab / kPubSlots) & 1u, ab)) break;
-        __threadfence();
-        atomicAdd(a.counters + slab, 1u);
       }
     }
   } else if (warp >= 4) {
@@ -640,7 +593,15 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       for (int visit = 0; ok && visit < 2; ++visit) {
         const int slab = visit == 0 ? t : t - a.lag;
         if (slab < 0 || slab >= n_slabs) continue;
-        // tile loop shared by both visits: the TMEM load of tile lt + 1 is in flight while tile lt is processed
+        // this run's row offsets (reference or lse) of the thread's columns
+        const int x = visit * 2 + (slab & 1);
+        if (!(ok = mbar_wait_warp(bars.o_ready(x), (uint32_t)(slab >> 1) & 1u, ab))) break;
+        float off[CH];
+#pragma unroll
+        for (int j = 0; j < CH; ++j) off[j] = rowoff[x * 64 + hh * CH + j];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars.o_free(x));
+        // tile loop shared by both visits
         float sum[CH];
 #pragma unroll
         for (int j = 0; j < CH; ++j) sum[j] = 0.f;
@@ -650,16 +611,16 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
             const int64_t key = (int64_t)(cta + lt * n_cta) * kTileKeys + quad * 32 + lane;
             if (key < a.n_tokens) {
 #pragma unroll
-              for (int j = 0; j < CH; ++j) sum[j] += fast_exp2(__uint_as_float(r[j]) * a.c);
+              for (int j = 0; j < CH; ++j) sum[j] += fast_exp2(fmaf(__uint_as_float(r[j]), a.c, -off[j]));
             }
           } else {
             // visit 2: running max over (layer, head) of q.k - lse/c
             float* slot = amax + ((int64_t)lt * NI + hh * (CH / G)) * kTileKeys + quad * 32 + lane;
 #pragma unroll
             for (int ii = 0; ii < CH / G; ++ii) {
-              float mx = __uint_as_float(r[ii * G]);
+              float mx = __uint_as_float(r[ii * G]) - off[ii * G];
 #pragma unroll
-              for (int g = 1; g < G; ++g) mx = fmaxf(mx, __uint_as_float(r[ii * G + g]));
+              for (int g = 1; g < G; ++g) mx = fmaxf(mx, __uint_as_float(r[ii * G + g]) - off[ii * G + g]);
               if (hh * (CH / G) + ii < a.n_lookahead) slot[ii * kTileKeys] = fmaxf(slot[ii * kTileKeys], mx);
             }
           }
@@ -677,17 +638,11 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
           if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));   // the stage can be overwritten: its data is in registers
           tr.advance();
         };
-        uint32_t ra[CH], rb[CH];
-        if (!(ok = start_load(ra))) break;
-        for (int lt = 0; lt < my_tiles; lt += 2) {
-          finish_load(ra);
-          if (lt + 1 < my_tiles && !(ok = start_load(rb))) break;
-          process(ra, lt);
-          if (lt + 1 < my_tiles) {
-            finish_load(rb);
-            if (lt + 2 < my_tiles && !(ok = start_load(ra))) break;
-            process(rb, lt + 1);
-          }
+        for (int lt = 0; lt < my_tiles; ++lt) {
+          uint32_t r[CH];
+          if (!(ok = start_load(r))) break;
+          finish_load(r);
+          process(r, lt);
         }
         if (!ok) break;
         if (visit == 0) {
@@ -805,7 +760,7 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
   pl.n_tiles = (int)ceil_div(p.n_tokens, kTileKeys);
   pl.n_cta = std::min(std::min(sm_count, kFusedMaxCtas), pl.n_tiles);
   pl.tiles_per_cta_max = (int)ceil_div(pl.n_tiles, pl.n_cta);
-  for (int ks = 8; ks >= 3; --ks) {
+  for (int ks = 10; ks >= 3; --ks) {
     const SmemLayout lay = smem_layout(p.head_dim, pl.ncols, g, ks, pl.tiles_per_cta_max);
     if ((int)lay.total <= kSmemBudget) {
       pl.k_stages = ks;

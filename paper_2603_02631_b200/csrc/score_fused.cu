@@ -273,6 +273,11 @@ __device__ __forceinline__ void tmem_wait<32>(uint32_t (&r)[32]) {
 }
 
 // ---------------------------------------------------------------------------------------------- layout
+// Key tiles per pipeline stage.  Every barrier hand-over (TMA -> MMA -> epilogue) and every tcgen05.commit costs
+// the issuing thread a few hundred cycles; with 64-wide heads a 128-key tile is only four small MMAs, so two
+// tiles travel together through the pipeline there.
+__host__ __device__ constexpr int group_tiles(int d) { return d == 64 ? 2 : 1; }
+
 struct SmemLayout {
   uint32_t k_off, q_off, amax_off, ref_off, rowoff_off, bar_off, misc_off, total;
 };
@@ -280,7 +285,7 @@ struct SmemLayout {
 __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, int k_stages, int tiles_per_cta_max) {
   SmemLayout s;
   uint32_t o = 0;
-  s.k_off = o;        o += (uint32_t)k_stages * (d / 64) * kSubTileBytes;
+  s.k_off = o;        o += (uint32_t)k_stages * group_tiles(d) * (d / 64) * kSubTileBytes;
   s.q_off = o;        o += (uint32_t)kQStages * (d / 64) * kQSubTileBytes;
   s.amax_off = o;     o += (uint32_t)tiles_per_cta_max * (ncols / group) * kTileKeys * 4;
   s.ref_off = o;      o += kRefSlots * 64 * 4;
@@ -342,6 +347,9 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   constexpr int CH = NCOLS / 2;          // query rows (TMEM columns) per epilogue thread
   constexpr int NI = NCOLS / G;          // lookahead slots per key in the running-max array
   constexpr int KSUB = D / 64;           // 64-wide sub-tiles per key tile
+  constexpr int GRP = group_tiles(D);    // key tiles per pipeline stage
+  constexpr int kStageBytes = GRP * KSUB * kSubTileBytes;
+  constexpr int kTmemCols = kTmemStages * GRP * NCOLS;
   static_assert(CH % G == 0, "a thread must own whole GQA groups");
 
   extern __shared__ unsigned char smem_raw[];
@@ -395,7 +403,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   fence_async_smem();
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)&misc[1])),
-                 "r"(kTmemStages * NCOLS)
+                 "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -421,13 +429,16 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
             tma_load_4d(smem_u32(q_tiles + (qr.stage * KSUB + h) * kQSubTileBytes), &maps.q, h * 64, 0, 0, slab,
                         bars.q_full(qr.stage));
           qr.advance();
-          for (int lt = 0; lt < my_tiles; ++lt) {
+          for (int lt0 = 0; lt0 < my_tiles; lt0 += GRP) {
+            const int n = min(GRP, my_tiles - lt0);
             if (!(ok = mbar_wait(bars.k_empty(kr.stage), kr.phase ^ 1u, ab))) break;
-            mbar_expect_tx(bars.k_full(kr.stage), (uint32_t)(KSUB * kSubTileBytes));
-            const int key0 = (cta + lt * n_cta) * kTileKeys;
-            for (int h = 0; h < KSUB; ++h)
-              tma_load_3d(smem_u32(k_tiles + (kr.stage * KSUB + h) * kSubTileBytes), &maps.k[layer], h * 64, key0, hk,
-                          bars.k_full(kr.stage));
+            mbar_expect_tx(bars.k_full(kr.stage), (uint32_t)(n * KSUB * kSubTileBytes));
+            for (int j = 0; j < n; ++j) {
+              const int key0 = (cta + (lt0 + j) * n_cta) * kTileKeys;
+              for (int h = 0; h < KSUB; ++h)
+                tma_load_3d(smem_u32(k_tiles + kr.stage * kStageBytes + (j * KSUB + h) * kSubTileBytes), &maps.k[layer],
+                            h * 64, key0, hk, bars.k_full(kr.stage));
+            }
             kr.advance();
           }
         }
@@ -449,22 +460,28 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
           if (slab < 0 || slab >= n_slabs) continue;
           if (!(ok = mbar_wait_warp(bars.q_full(qr.stage), qr.phase, ab))) break;
           const uint64_t bd0 = q_desc0 + (uint64_t)((qr.stage * KSUB * kQSubTileBytes) >> 4);
-          for (int lt = 0; lt < my_tiles; ++lt) {
-            if (lt % kIssuers == me) {
+          for (int lt0 = 0, grp = 0; lt0 < my_tiles; lt0 += GRP, ++grp) {
+            if (grp % kIssuers == me) {
+              const int n = min(GRP, my_tiles - lt0);
               if (!(ok = mbar_wait_warp(bars.k_full(kr.stage), kr.phase, ab))) break;
               if (!(ok = mbar_wait_warp(bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
               tc_fence_after();
-              const uint32_t d_tmem = tmem_base + (uint32_t)(tr.stage * NCOLS);
-              const uint64_t ad0 = k_desc0 + (uint64_t)((kr.stage * KSUB * kSubTileBytes) >> 4);
+              const uint32_t d_tmem = tmem_base + (uint32_t)(tr.stage * GRP * NCOLS);
+              const uint64_t ad0 = k_desc0 + (uint64_t)((kr.stage * kStageBytes) >> 4);
               if (elect_one()) {
 #pragma unroll
-                for (int h = 0; h < KSUB; ++h) {
+                for (int j = 0; j < GRP; ++j) {
+                  if (j < n) {
 #pragma unroll
-                  for (int ks = 0; ks < 4; ++ks)
-                    tc_mma(d_tmem, ad0 + (uint64_t)((h * kSubTileBytes) >> 4) + 2u * ks,
-                           bd0 + (uint64_t)((h * kQSubTileBytes) >> 4) + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
+                    for (int h = 0; h < KSUB; ++h) {
+#pragma unroll
+                      for (int ks = 0; ks < 4; ++ks)
+                        tc_mma(d_tmem + (uint32_t)(j * NCOLS), ad0 + (uint64_t)(((j * KSUB + h) * kSubTileBytes) >> 4) + 2u * ks,
+                               bd0 + (uint64_t)((h * kQSubTileBytes) >> 4) + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
+                    }
+                  }
                 }
-                tc_commit(bars.k_empty(kr.stage));
+                tc_commit(bars.k_empty(kr.stage));             // one pair of commits per stage, however many tiles
                 tc_commit(bars.t_full(tr.stage));
               }
               __syncwarp();
@@ -625,24 +642,27 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
             }
           }
         };
-        auto start_load = [&](uint32_t (&r)[CH]) -> bool {
-          if (!mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab)) return false;
+        for (int lt0 = 0; lt0 < my_tiles; lt0 += GRP) {
+          const int n = min(GRP, my_tiles - lt0);
+          if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
           tc_fence_after();
-          tmem_issue<CH>(tmem_base + lane_addr + (uint32_t)(tr.stage * NCOLS + hh * CH), r);
-          return true;
-        };
-        auto finish_load = [&](uint32_t (&r)[CH]) {
-          tmem_wait<CH>(r);
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));   // the stage can be overwritten: its data is in registers
+          const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(tr.stage * GRP * NCOLS + hh * CH);
+#pragma unroll
+          for (int j = 0; j < GRP; ++j) {
+            if (j < n) {
+              uint32_t r[CH];
+              tmem_issue<CH>(taddr + (uint32_t)(j * NCOLS), r);
+              tmem_wait<CH>(r);
+              if (j == n - 1) {
+                // the stage can be overwritten: its last tile is in registers
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
+              }
+              process(r, lt0 + j);
+            }
+          }
           tr.advance();
-        };
-        for (int lt = 0; lt < my_tiles; ++lt) {
-          uint32_t r[CH];
-          if (!(ok = start_load(r))) break;
-          finish_load(r);
-          process(r, lt);
         }
         if (!ok) break;
         if (visit == 0) {
@@ -718,7 +738,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   __syncthreads();
   if (warp == 0) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemStages * NCOLS) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -760,7 +780,7 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
   pl.n_tiles = (int)ceil_div(p.n_tokens, kTileKeys);
   pl.n_cta = std::min(std::min(sm_count, kFusedMaxCtas), pl.n_tiles);
   pl.tiles_per_cta_max = (int)ceil_div(pl.n_tiles, pl.n_cta);
-  for (int ks = 10; ks >= 3; --ks) {
+  for (int ks = 10; ks >= 2; --ks) {
     const SmemLayout lay = smem_layout(p.head_dim, pl.ncols, g, ks, pl.tiles_per_cta_max);
     if ((int)lay.total <= kSmemBudget) {
       pl.k_stages = ks;

@@ -353,7 +353,9 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   static_assert(CH % G == 0, "a thread must own whole GQA groups");
 
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // 1024-byte alignment by offsetting the shared array itself, so that the compiler still knows these are
+  // shared-memory addresses (a round trip through an integer would turn every access into a generic one)
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const SmemLayout lay = smem_layout(D, NCOLS, G, a.k_stages, a.tiles_per_cta_max);
   unsigned char* k_tiles = smem + lay.k_off;
   unsigned char* q_tiles = smem + lay.q_off;

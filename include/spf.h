@@ -117,6 +117,14 @@ SPF_API int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int
 SPF_API int32_t spf_set_score_path(int32_t path);
 
 /*
+ * Diagnostic (no counterpart in the paper): checks that a device-side wait of the fused kernel gives up
+ * instead of hanging.  Enqueues a one-CTA kernel that waits, with the kernels' own bounded wait and a
+ * 20 ms limit, on a barrier nothing ever signals.  After synchronising, *dev_status (device int32, zeroed
+ * by the caller) must read SPF_ERR_TIMEOUT and the context must still be usable.
+ */
+SPF_API int32_t spf_selftest_bounded_wait(int32_t* dev_status, void* cuda_stream);
+
+/*
  * spf_score without a caller-provided workspace (the paper has no counterpart; this exists for
  * deployment reasons only).
  *

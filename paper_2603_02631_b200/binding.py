@@ -44,6 +44,8 @@ def _load() -> ctypes.CDLL:
     dll.spf_score_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32]
     dll.spf_score.restype = i32
     dll.spf_score.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp, ctypes.c_size_t, vp, vp]
+    dll.spf_selftest_bounded_wait.restype = i32
+    dll.spf_selftest_bounded_wait.argtypes = [vp, vp]
     dll.spf_set_score_path.restype = i32
     dll.spf_set_score_path.argtypes = [i32]
     dll.spf_score_static.restype = i32
@@ -162,6 +164,12 @@ def spf_score(prompts: Sequence[PromptBuffers], workspace: torch.Tensor, softmax
     _check(lib.spf_score(ctypes.byref(shape), arr, len(prompts), workspace.data_ptr(),
                          workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
            "spf_score")
+
+
+def spf_selftest_bounded_wait(dev_status: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Enqueues the bounded-wait self-test; dev_status (int32, zeroed) reads SPF_ERR_TIMEOUT (-5) afterwards."""
+    _dev(dev_status, torch.int32, "dev_status")
+    _check(lib.spf_selftest_bounded_wait(dev_status.data_ptr(), _stream_ptr(stream)), "spf_selftest_bounded_wait")
 
 
 def spf_set_score_path(path: int) -> int:
@@ -298,6 +306,29 @@ class Selector:
         L, Hq, _, _, m = self.geom
         return Selection(self.importance[:n], self.lse.view(L, Hq, m), self.chunk_scores[:n_chunks], k, self.kept,
                          self.out_ids, self.out_pos, self.tok_spans, self.char_spans, self.counts)
+
+    def run_checked(self, q: torch.Tensor, k_layers: Sequence[torch.Tensor], token_ids: torch.Tensor,
+                    char_start: torch.Tensor, char_end: torch.Tensor, keep: float,
+                    stream: Optional[torch.cuda.Stream] = None) -> Selection:
+        """Like run(), but synchronises and reads the device status.  If the fused scoring kernel reported
+        SPF_ERR_RANGE (a logit beyond its fp32 guard), the prompt is scored again on the general path, which
+        has no such limit.  Any other device status raises."""
+        self.dev_status.zero_()
+        sel = self.run(q, k_layers, token_ids, char_start, char_end, keep, stream)
+        (stream or torch.cuda.current_stream()).synchronize()
+        status = int(self.dev_status.item())
+        if status == -6:
+            previous = spf_set_score_path(1)
+            try:
+                self.dev_status.zero_()
+                sel = self.run(q, k_layers, token_ids, char_start, char_end, keep, stream)
+                (stream or torch.cuda.current_stream()).synchronize()
+                status = int(self.dev_status.item())
+            finally:
+                spf_set_score_path(previous)
+        if status != 0:
+            raise SpfError(status, "Selector.run_checked", spf_status_string(status))
+        return sel
 
     def run_host(self, q: torch.Tensor, k_layers: Sequence[torch.Tensor], token_ids: torch.Tensor,
                  char_start: torch.Tensor, char_end: torch.Tensor, keep: float):

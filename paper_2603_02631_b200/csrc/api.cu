@@ -146,6 +146,12 @@ extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, 
   return SPF_OK;
 }
 
+extern "C" int32_t spf_selftest_bounded_wait(int32_t* dev_status, void* cuda_stream) {
+  clear_error();
+  if (dev_status == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_selftest_bounded_wait: dev_status is null");
+  return bounded_wait_selftest_launch(dev_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
 extern "C" int32_t spf_set_score_path(int32_t path) {
   if (path < 0 || path > 2) return g_score_path.load(std::memory_order_relaxed);
   return g_score_path.exchange(path, std::memory_order_relaxed);

@@ -31,4 +31,7 @@ bool score_fused_supported(const ScoreProblem& p, int sm_count);
 size_t score_fused_workspace_bytes(const ScoreProblem& p);
 int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count, int32_t* dev_status, cudaStream_t stream);
 
+// Launches the one-CTA self-test of the kernels' bounded wait (see spf_selftest_bounded_wait).
+int32_t bounded_wait_selftest_launch(int32_t* dev_status, cudaStream_t stream);
+
 }  // namespace spf

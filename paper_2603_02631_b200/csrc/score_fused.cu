@@ -111,6 +111,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 struct Abort {
   volatile int* flag;      // shared: set once any wait of this CTA ran out
   int32_t* dev_status;     // global, may be null
+  unsigned long long timeout_ns = kTimeoutNs;   // how long a single wait may last
 };
 
 __device__ __noinline__ void record_timeout(const Abort& ab) {
@@ -128,7 +129,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
       if (*ab.flag) return false;
       const unsigned long long now = global_timer();
       if (t0 == 0) t0 = now;
-      if (now - t0 > kTimeoutNs) {
+      if (now - t0 > ab.timeout_ns) {
         record_timeout(ab);
         return false;
       }
@@ -153,7 +154,7 @@ __device__ __forceinline__ bool count_wait(const unsigned* counter, unsigned tar
       if (*ab.flag) return false;
       const unsigned long long now = global_timer();
       if (t0 == 0) t0 = now;
-      if (now - t0 > kTimeoutNs) {
+      if (now - t0 > ab.timeout_ns) {
         record_timeout(ab);
         return false;
       }
@@ -852,6 +853,28 @@ int32_t launch_fused_n(int ncols, int g, const FusedMaps& maps, const FusedArgs&
 }
 
 }  // namespace
+
+// One CTA waits on an mbarrier that nothing ever arrives on, with the kernels' own bounded wait and a
+// 20 ms limit: the wait must give up, record SPF_ERR_TIMEOUT and let the kernel return normally.
+__global__ void bounded_wait_selftest_kernel(int32_t* dev_status) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const Abort ab{&abort_flag, dev_status, 20000000ull};
+  mbar_wait_warp(smem_u32(&bar), 0u, ab);
+  __syncthreads();
+}
+
+int32_t bounded_wait_selftest_launch(int32_t* dev_status, cudaStream_t stream) {
+  bounded_wait_selftest_kernel<<<1, 64, 0, stream>>>(dev_status);
+  SPF_CUDA_CHECK(cudaGetLastError());
+  return SPF_OK;
+}
 
 bool score_fused_supported(const ScoreProblem& p, int sm_count) { return make_plan(p, sm_count).ok; }
 

@@ -186,6 +186,29 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------------------------- multi-rank helpers
+def rank_config(cfg, rank):
+    """Weak scaling: every rank gets the same shapes and its own prompts (a different seed per rank)."""
+    import dataclasses
+    return cfg if rank == 0 else dataclasses.replace(cfg, seed=cfg.seed + 1000 * rank)
+
+
+def max_over_ranks(values, device, world):
+    """Element-wise maximum over all ranks of a list of floats (identity for a single process)."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(tokens_per_rank_step, steps, world, ms_total_max):
+    """Aggregate tokens per second of all ranks: every rank processed the same number of tokens."""
+    return world * tokens_per_rank_step * steps / (ms_total_max * 1e-3)
+
+
 # ----------------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -206,9 +229,7 @@ def run_ours(args):
     keep = cfg.keep[0]
     n_prompts = len(cfg.lengths)
     # weak scaling: every rank gets the same shapes, its own prompts (distinct seeds via the prompt index)
-    prompts = [make_prompt(cfg, i, dev) if rank == 0 else
-               make_prompt(__import__("dataclasses").replace(cfg, seed=cfg.seed + 1000 * rank), i, dev)
-               for i in range(n_prompts)]
+    prompts = [make_prompt(rank_config(cfg, rank), i, dev) for i in range(n_prompts)]
     max_n = max(cfg.lengths)
     sel = spf.Selector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, max_n,
                        chunk=cfg.chunk, pool_kernel=cfg.pool_kernel, device=dev)
@@ -307,18 +328,15 @@ def run_ours(args):
         e2e = {"seconds": e2e_s, "h2d": h2d, "d2h": d2h}
 
     # --- reduce over ranks --------------------------------------------------------------------------
-    if world > 1:
-        t = torch.tensor([ms_total, e2e["seconds"] if e2e else 0.0, score_ms_avg], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, e2e_s_max, score_ms_avg = t.tolist()
-        if e2e:
-            e2e["seconds"] = e2e_s_max
+    ms_total, e2e_s_max, score_ms_avg = max_over_ranks([ms_total, e2e["seconds"] if e2e else 0.0, score_ms_avg], dev, world)
+    if e2e:
+        e2e["seconds"] = e2e_s_max
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    value = world * tokens_per_step * args.steps / (ms_total * 1e-3)
+    value = whole_job_value(tokens_per_step, args.steps, world, ms_total)
     peak, peak_kind = hbm_peak()
     k_bytes = cfg.k_bytes()
     q_bytes = n_prompts * cfg.n_layers * cfg.n_q_heads * cfg.n_lookahead * cfg.head_dim * 2

@@ -31,6 +31,29 @@ DEFAULT_WORKLOAD = "long128k"          # N = 131072, the configuration the metri
 FALLBACK_HBM_GBS = 6650.0
 
 
+# DRAM read + write bytes of one scoring launch, from the ncu capture summarised in profiles/.  Each entry names
+# the SHA-256 of the kernel source it was taken from: once the source changes, the figure is reported as null.
+NCU_TRAFFIC = {
+    ("long128k", "fused"): {"bytes": 4 * (577388800 + 4997888), "source": "paper_2603_02631_b200/csrc/score_fused.cu",
+                            "sha256": "4cd2cf848a3385c571ae6f75bc18658e97335a9db49d71f51a28df4e49d0305e",
+                            "note": "captured on long128k_l4 (4 of 16 layers), scaled x4"},
+}
+
+
+def ncu_traffic(workload, path):
+    import hashlib
+    entry = NCU_TRAFFIC.get((workload, path))
+    if entry is None:
+        return None
+    try:
+        with open(os.path.join(ROOT, entry["source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != entry["sha256"]:
+                return None
+    except OSError:
+        return None
+    return entry["bytes"]
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -356,7 +379,7 @@ def run_ours(args):
         "gpu_launches": launches_per_prompt * n_prompts * args.steps,
         "roofline": {"bound": "hbm", "kernel": f"spf_score ({score_kernels})",
                      "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None, "ms_per_launch": score_ms_avg,
+                     "frac": achieved / peak, "traffic": ncu_traffic(cfg.name, "fused" if fused else "general"), "ms_per_launch": score_ms_avg,
                      "algorithmic_bytes": score_bytes},
     }
     if e2e:

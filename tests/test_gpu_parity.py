@@ -215,3 +215,17 @@ def test_determinism_across_runs(spf):
         again = gpu_run(prompt, 0.1)
         assert np.array_equal(first["importance"], again["importance"])
         assert np.array_equal(first["kept"], again["kept"])
+
+
+def test_host_buffer_entry_matches_device_entry(spf):
+    """Selector.run_host (pinned host tensors in, host arrays out) gives what Selector.run gives on device tensors."""
+    cfg = small_config("host", n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, n_lookahead=8, lengths=(3000,), seed=8)
+    prompt = make_prompt(cfg)
+    sel = spf.Selector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, prompt.n_tokens,
+                       chunk=cfg.chunk, pool_kernel=cfg.pool_kernel)
+    pin = lambda t: t.pin_memory()
+    host = sel.run_host(pin(prompt.q), [pin(x) for x in prompt.k], pin(prompt.token_ids), pin(prompt.char_start),
+                        pin(prompt.char_end), 0.2)
+    dev = gpu_run(prompt, 0.2, sel)
+    for key in ("ids", "pos", "tok_spans", "char_spans"):
+        assert np.array_equal(host[key], dev[key])

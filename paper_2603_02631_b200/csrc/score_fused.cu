@@ -47,12 +47,10 @@ namespace spf {
 namespace {
 
 constexpr int kTileKeys = 128;
-constexpr int kThreads = 384;          // warp 0 TMA, 1 MMA issue, 2 control, 3 publisher, 4..11 epilogue
+constexpr int kThreads = 640;          // warp 0 TMA, 1 MMA issue, 2 control, 3 publisher, 4..19 epilogue
 constexpr int kIssuers = 1;            // MMA-issuing warps: local tile lt belongs to issuer lt % kIssuers
 constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accumulators (covers every finite fp32)
 constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
-constexpr int kEpiWarps = 8;
-constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kQStages = 3;
 constexpr int kTmemStages = 4;
 constexpr int kRefSlots = 8;
@@ -328,7 +326,7 @@ struct Ring {
   }
 };
 
-// Barrier among the eight epilogue warps, with a bounded wait (an mbarrier with one arrival per warp).
+// Barrier among the epilogue warps, with a bounded wait (an mbarrier with one arrival per warp).
 struct EpiSync {
   uint32_t bar;
   uint32_t phase = 0;
@@ -345,7 +343,9 @@ struct EpiSync {
 template <int D, int NCOLS, int G>
 __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_constant__ FusedMaps maps,
                                                                    const __grid_constant__ FusedArgs a) {
-  constexpr int CH = NCOLS / 2;          // query rows (TMEM columns) per epilogue thread
+  constexpr int NSPLIT = NCOLS >= 64 ? 4 : 2;   // epilogue warps per TMEM lane quadrant: each takes a slice of the columns
+  constexpr int EW = 4 * NSPLIT;                // epilogue warps: 16 or 8
+  constexpr int CH = NCOLS / NSPLIT;            // query rows (TMEM columns) per epilogue thread: 16 or 8
   constexpr int NI = NCOLS / G;          // lookahead slots per key in the running-max array
   constexpr int KSUB = D / 64;           // 64-wide sub-tiles per key tile
   constexpr int GRP = group_tiles(D);    // key tiles per pipeline stage
@@ -388,15 +388,15 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     }
     for (int s = 0; s < kTmemStages; ++s) {
       mbar_init(bars.t_full(s), 1);
-      mbar_init(bars.t_empty(s), kEpiWarps);
+      mbar_init(bars.t_empty(s), EW);
     }
     for (int x = 0; x < 4; ++x) {
       mbar_init(bars.o_ready(x), 1);
-      mbar_init(bars.o_free(x), kEpiWarps);
+      mbar_init(bars.o_free(x), EW);
     }
-    mbar_init(bars.epi_sync(), kEpiWarps);
+    mbar_init(bars.epi_sync(), EW);
     mbar_init(bars.mma_done(), kIssuers);
-    for (int b = 0; b < kPubSlots; ++b) mbar_init(bars.pub_ready(b), kEpiWarps);
+    for (int b = 0; b < kPubSlots; ++b) mbar_init(bars.pub_ready(b), EW);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // zero the query stages: rows the TMA box does not cover must read as zero
@@ -506,7 +506,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       }
     }
   } else if (warp == 3) {
-    // ===== publisher: once the eight epilogue warps have added their shares of a slab's row sums, order those
+    // ===== publisher: once the epilogue warps have added their shares of a slab's row sums, order those
     // additions before the arrival count and report this CTA (keeps the fence off the epilogue warps) =====
     if (lane == 0) {
       for (int slab = 0; slab < n_slabs; ++slab) {
@@ -600,11 +600,12 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         if (lane == 0) mbar_arrive(bars.o_ready(x));
       }
     }
-  } else if (warp >= 4) {
-    // ===== epilogue: 8 warps; warp % 4 picks the TMEM lane quadrant (keys), warps 4-7 / 8-11 the column half =====
+  } else if (warp >= 4 && warp < 4 + EW) {
+    // ===== epilogue: EW warps; warp % 4 picks the TMEM lane quadrant (32 keys), (warp - 4) / 4 the slice of CH columns.
+    // With 64 query rows four warps share a quadrant: they hide each other's barrier and TMEM-load latencies =====
     const int quad = warp & 3;
     const int hh = (warp - 4) >> 2;
-    const int et = threadIdx.x - 128;                           // 0..255 among epilogue threads
+    const int et = threadIdx.x - 128;                           // index among the epilogue threads
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     Ring tr(kTmemStages);
     EpiSync es{bars.epi_sync()};
@@ -718,7 +719,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     if (ok) ok = es.sync(lane, ab);
     if (ok && misc[0] == 0) {
       const float inv_m = 1.f / (float)a.n_lookahead;
-      for (int idx = et; idx < my_tiles * kTileKeys; idx += kEpiThreads) {
+      for (int idx = et; idx < my_tiles * kTileKeys; idx += EW * 32) {
         const int lt = idx / kTileKeys, kk = idx % kTileKeys;
         const int64_t key = (int64_t)(cta + lt * n_cta) * kTileKeys + kk;
         if (key < a.n_tokens) {

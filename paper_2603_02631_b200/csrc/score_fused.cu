@@ -53,7 +53,7 @@ constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accu
 constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
 constexpr int kQStages = 3;
 constexpr int kTmemStages = 4;
-constexpr int kRefSlots = 8;
+constexpr int kRefSlots = 16;         // row references stay readable for this many slabs (must exceed the lag)
 constexpr int kPubSlots = 4;
 constexpr float kRefMargin = 60.f;     // base-2 units added to the sampled reference logit
 constexpr unsigned long long kTimeoutNs = 2000000000ull;
@@ -796,13 +796,17 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
   return pl;
 }
 
-// How many slabs the second visit runs behind the first.  Two leaves a full slab of time for the
-// cross-CTA merge of the row sums; the environment variable SPF_FUSED_LAG (1..4) overrides it for tuning.
-int fused_lag(int n_slabs) {
-  int lag = 2;
+// How many slabs the second visit runs behind the first.  The cross-CTA hand-over of a slab's row sums takes
+// about 5 us; with short slabs (few tiles per CTA) two slabs of lead do not cover it, so the lag grows until the
+// slabs kept live for the second read (lag + 1 of them) would no longer sit comfortably in L2.  The
+// environment variable SPF_FUSED_LAG (1..8) overrides the choice for tuning.
+int fused_lag(const ScoreProblem& p, int n_slabs) {
+  const double slab_bytes = (double)p.n_tokens * p.head_dim * 2.0;
+  int lag = (int)(40.0 * 1024 * 1024 / slab_bytes) - 1;
+  lag = std::max(2, std::min(lag, 8));
   if (const char* env = getenv("SPF_FUSED_LAG")) {
     const int v = atoi(env);
-    if (v >= 1 && v <= 4) lag = v;
+    if (v >= 1 && v <= 8) lag = v;
   }
   return std::max(1, std::min(lag, n_slabs));
 }
@@ -926,7 +930,7 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   args.n_lookahead = m;
   args.n_tiles = pl.n_tiles;
   args.tiles_per_cta_max = pl.tiles_per_cta_max;
-  args.lag = fused_lag(n_slabs);
+  args.lag = fused_lag(p, n_slabs);
   args.k_stages = pl.k_stages;
   args.c = p.c_log2;
   args.inv_c = 1.0f / p.c_log2;

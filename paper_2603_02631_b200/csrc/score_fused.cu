@@ -123,6 +123,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
   unsigned long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (it > 2u) __nanosleep(64);   // do not poll hot next to the warps that do the arithmetic
     if ((it & 63u) == 0u) {
       if (*ab.flag) return false;
       const unsigned long long now = global_timer();

@@ -309,14 +309,16 @@ def run_ours(args):
     score_ms = []
     bufs = [spf.binding.PromptBuffers(p.q, p.k, sel.importance[:p.n_tokens], sel.lse) for p in prompts]
     ws = sel._workspace(bufs[cfg.lengths.index(max_n)])
+    events = []
     for it in range(args.steps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
         for bf in bufs:
             spf.spf_score([bf], ws, 0.0, sel.dev_status)
         b.record(stream)
-        b.synchronize()
-        score_ms.append(a.elapsed_time(b))
+        events.append((a, b))
+    torch.cuda.synchronize()
+    score_ms = [a.elapsed_time(b) for a, b in events]
     score_ms_avg = sum(score_ms) / len(score_ms)
 
     # --- end to end from pinned host memory -----------------------------------------------------

@@ -81,14 +81,40 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
       if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      int rem = remaining, b = 255;
-      for (; b > 0; --b) {
-        if (hist[b] >= rem) break;
-        rem -= hist[b];
+    if (threadIdx.x < 32) {
+      // warp 0 walks the 256 bins from the top: each lane owns 8 consecutive bins (lane 31 the highest)
+      const int lane = threadIdx.x;
+      int mine[8], own = 0;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        mine[e] = hist[lane * 8 + e];
+        own += mine[e];
       }
-      sh_prefix = prefix | ((uint32_t)b << shift);
-      sh_remaining = rem;
+      int above = own;                                   // inclusive suffix sum over lanes >= this one
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int v = __shfl_down_sync(0xffffffffu, above, off);
+        if (lane + off < 32) above += v;
+      }
+      above -= own;                                      // entries in bins owned by higher lanes
+      const bool here = above < remaining && above + own >= remaining;   // the wanted rank falls into this lane's bins
+      if (here) {
+        int rem = remaining - above, b = 0;
+        bool found = false;
+#pragma unroll
+        for (int e = 7; e >= 0; --e) {
+          if (!found) {
+            if (mine[e] >= rem || e == 0) {
+              b = e;
+              found = true;
+            } else {
+              rem -= mine[e];
+            }
+          }
+        }
+        sh_prefix = prefix | ((uint32_t)(lane * 8 + b) << shift);
+        sh_remaining = rem;
+      }
     }
     __syncthreads();
     prefix = sh_prefix;

@@ -42,6 +42,8 @@ SHAPES = [
     (1, 4, 2, 128, 12, 1500, 128),         # m=12 padded to 16, chunk 128
     (1, 2, 1, 64, 20, 900, 32),            # m=20 padded to 24
     (1, 2, 1, 64, 32, 650, 32),            # m=32
+    (1, 2, 1, 128, 8, 60001, 32),          # d=128, four one-tile pipeline stages per CTA in the fused path
+    (1, 4, 1, 64, 16, 50000, 32),          # d=64, 64 query rows, three tiles (two stages, the second half full) per CTA
     (2, 4, 2, 64, 8, 31, 32),              # a single partial key tile and a single chunk
     (1, 1, 1, 64, 8, 1, 32),               # one token
 ]

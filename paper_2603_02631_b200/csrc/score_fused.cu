@@ -5,9 +5,9 @@
 // keys of the row.  Each (layer, kv-head) slab of keys is therefore visited twice:
 //   visit 1 ("sum")  accumulates  sum_s exp2(c * q.k - ref)  per query row;
 //   visit 2 ("max")  folds  max_{l,h} (q.k - lse/c)  into a running maximum per (lookahead i, key s).
-// The kernel software-pipelines the two visits by `lag` slabs: while slab t streams in from HBM for
-// visit 1, slab t - lag is read again for visit 2 -- by the same CTA that read it a few microseconds
-// earlier, so the second read is served by L2.
+// The two visits are software-pipelined `lag` slabs apart and travel TOGETHER through the pipeline: stage
+// (t, j) holds tile j of slab t for visit 1 (streamed from HBM, kept in L2 with an evict-last hint) and
+// tile j of slab t - lag for visit 2 (read again by the same CTA, so from L2, with an evict-first hint).
 //
 // Work split.  The grid is persistent (one CTA per SM).  CTA b owns key tiles b, b + grid, ... (128
 // keys each) of EVERY slab, so its running maxima for those keys stay in its shared memory for the
@@ -16,21 +16,27 @@
 // One tile = one tcgen05 MMA group: A = 128 keys x d (shared memory, TMA, 128-byte swizzle),
 // B = the slab's query rows x d (row j = i * G + g: lookahead i, head g of the GQA group), D = fp32
 // [128 keys x NCOLS rows] in tensor memory.  Keys are TMEM lanes, so an epilogue thread owns one key
-// and sees all query rows of it: the max over heads is in-thread, and the sum over keys is kept
-// per thread and reduced across threads only once per slab.
+// and sees all query rows of it: the max over heads is in-thread.
 //
-// Row offsets.  Visit 1 subtracts a per-row reference ref (in base-2 units) inside the exp2 argument so that
-// exp2 cannot overflow: the reference of a row is its logit against one fixed sample key plus a margin of 60,
-// so sums stay finite unless some key beats the sample by more than 2^187 (then the row's sum becomes inf and
-// SPF_ERR_RANGE is reported).  Visit 2 subtracts lse/c.  A control warp prepares both per slab in shared memory.
+// Warps.  0: TMA producer.  1: MMA issuer.  2: log-sum-exp warp (turns a slab's complete row sums into the
+// offsets of visit 2).  3: reference + publisher warp.  4..11: "sum" warps, the visit-1 half of every stage
+// (exp2-bound).  12..19: "max" warps, the visit-2 half (ALU / shared-memory bound); they also add up the per-key
+// sums of the sum warps, which reach them through a shared-memory buffer once per slab.  The two groups run
+// independently, so the exp2 work and the max work overlap on every scheduler.
 //
-// Cross-CTA step.  All CTAs use the same reference for a row (its logit against one fixed sample key),
-// so their partial sums can simply be added.  To make the total independent of the order in which
-// CTAs arrive, the fp32 partial sums are added EXACTLY: each is split over two 40-bit limbs of a
-// 280-bit fixed-point accumulator per row (64-bit integer atomics, no carries needed), which covers
-// every finite fp32 value.  A counter per slab tells the visit-2 side of every CTA when all shares
-// are in; it then converts the accumulator to lse itself.  Results are bit-identical from run to run.
-// Because visit 1 never waits on another CTA and all CTAs are co-resident, the counters always fill.
+// Reference.  Visit 1 subtracts one reference per slab inside the exp2 argument so that exp2 cannot overflow:
+// the largest logit of the slab's rows against one fixed sample key, plus a margin of 60 (base-2 units).  Sums
+// stay finite unless some logit exceeds that sample logit by more than about 50 base-2 units; a row whose logits
+// all lie more than 186 units below it sums to zero.  Both cases are reported as SPF_ERR_RANGE (the caller can
+// then use the general path).
+//
+// Cross-CTA step.  All CTAs use the same reference for a slab, so their partial sums can simply be added.
+// To make the total independent of the order in which CTAs arrive, the fp32 partial sums are added
+// EXACTLY: each is split over two 40-bit limbs of a 280-bit fixed-point accumulator per row (64-bit integer
+// atomics, no carries needed), which covers every finite fp32 value.  A counter per slab tells the
+// log-sum-exp warp of every CTA when all shares are in; it then converts the accumulator to lse itself.
+// Results are bit-identical from run to run.  Because visit 1 never waits on another CTA and all CTAs are
+// co-resident, the counters always fill.
 //
 // Every wait in this file is bounded: on expiry the kernel records SPF_ERR_TIMEOUT, drains and
 // returns normally.
@@ -47,18 +53,17 @@ namespace spf {
 namespace {
 
 constexpr int kTileKeys = 128;
-constexpr int kThreads = 640;          // warp 0 TMA, 1 MMA issue, 2 control, 3 publisher, 4..19 epilogue
+constexpr int kThreads = 640;          // warp 0 TMA, 1 MMA issue, 2 log-sum-exp, 3 references + publisher, 4..19 epilogue
 constexpr int kIssuers = 1;            // MMA-issuing warps: local tile lt belongs to issuer lt % kIssuers
 constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accumulators (covers every finite fp32)
 constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
-constexpr int kQStages = 3;
+constexpr int kQStages = 2;
 constexpr int kTmemStages = 4;
 constexpr int kRefSlots = 16;         // row references stay readable for this many slabs (must exceed the lag)
-constexpr int kPubSlots = 4;
+constexpr int kPubSlots = 16;        // slabs whose hand-over to the publisher may be pending at once
 constexpr float kRefMargin = 60.f;     // base-2 units added to the sampled reference logit
 constexpr unsigned long long kTimeoutNs = 2000000000ull;
 constexpr int kSubTileBytes = kTileKeys * 128;  // 128 keys x 64 bf16, one swizzle-128B tile
-constexpr int kQSubTileBytes = 64 * 128;        // up to 64 query rows x 64 bf16
 
 struct FusedMaps {
   CUtensorMap q;                      // (d, g, i, slab) view of the query tensor
@@ -162,11 +167,46 @@ __device__ __forceinline__ bool count_wait(const unsigned* counter, unsigned tar
   }
 }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+
+// Waits until *flag (shared memory, written by another warp of the CTA) has reached `target`.
+__device__ __forceinline__ bool flag_wait(const volatile int* flag, int target, const Abort& ab) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (*flag >= target) {
+      __threadfence_block();
+      return true;
+    }
+    if ((it & 15u) == 15u) {
+      if (*ab.flag) return false;
+      const unsigned long long now = global_timer();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > ab.timeout_ns) {
+        record_timeout(ab);
+        return false;
+      }
+      __nanosleep(100);
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar,
+                                            uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy)
       : "memory");
+}
+// L2 eviction priorities for the key tiles: the first visit's tile is read again `lag` slabs later (keep it), the
+// second visit's tile is dead once it has been read (let it go first)
+__device__ __forceinline__ uint64_t l2_policy_keep() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_drop() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
                                             uint32_t bar) {
@@ -273,22 +313,20 @@ __device__ __forceinline__ void tmem_wait<32>(uint32_t (&r)[32]) {
 }
 
 // ---------------------------------------------------------------------------------------------- layout
-// Key tiles per pipeline stage.  Every barrier hand-over (TMA -> MMA -> epilogue) and every tcgen05.commit costs
-// the issuing thread a few hundred cycles; with 64-wide heads a 128-key tile is only four small MMAs, so two
-// tiles travel together through the pipeline there.
-__host__ __device__ constexpr int group_tiles(int d) { return d == 64 ? 2 : 1; }
+__host__ __device__ constexpr int q_sub_tile_bytes(int ncols) { return ncols * 128; }   // ncols query rows x 64 bf16
 
 struct SmemLayout {
-  uint32_t k_off, q_off, amax_off, ref_off, rowoff_off, bar_off, misc_off, total;
+  uint32_t k_off, q_off, amax_off, xbuf_off, ref_off, rowoff_off, bar_off, misc_off, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, int k_stages, int tiles_per_cta_max) {
   SmemLayout s;
   uint32_t o = 0;
-  s.k_off = o;        o += (uint32_t)k_stages * group_tiles(d) * (d / 64) * kSubTileBytes;
-  s.q_off = o;        o += (uint32_t)kQStages * (d / 64) * kQSubTileBytes;
+  s.k_off = o;        o += (uint32_t)k_stages * 2 * (d / 64) * kSubTileBytes;
+  s.q_off = o;        o += (uint32_t)kQStages * 2 * (d / 64) * q_sub_tile_bytes(ncols);
   s.amax_off = o;     o += (uint32_t)tiles_per_cta_max * (ncols / group) * kTileKeys * 4;
-  s.ref_off = o;      o += kRefSlots * 64 * 4;
+  s.xbuf_off = o;     o += (uint32_t)ncols * kTileKeys * 4;
+  s.ref_off = o;      o += kRefSlots * 4;
   s.rowoff_off = o;   o += 4 * 64 * 4;
   s.bar_off = o;      o += 64 * 8;
   s.misc_off = o;     o += 64;
@@ -311,8 +349,10 @@ struct Bars {
   __device__ uint32_t epi_sync() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 8); }
   __device__ uint32_t mma_done() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 9); }
   __device__ uint32_t pub_ready(int b) const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 10 + b); }
+  __device__ uint32_t x_ready() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 10 + kPubSlots); }
+  __device__ uint32_t x_free() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 11 + kPubSlots); }
 };
-// 2 * 10 + 2 * 3 + 2 * 4 + 14 = 48 barriers at most; the block has room for 64.
+// 2 * 10 + 2 * 2 + 2 * 4 + 10 + 16 + 2 = 60 barriers at most; the block has room for 64.
 
 struct Ring {
   int stage = 0;
@@ -344,15 +384,19 @@ struct EpiSync {
 template <int D, int NCOLS, int G>
 __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_constant__ FusedMaps maps,
                                                                    const __grid_constant__ FusedArgs a) {
-  constexpr int NSPLIT = NCOLS >= 64 ? 4 : 2;   // epilogue warps per TMEM lane quadrant: each takes a slice of the columns
-  constexpr int EW = 4 * NSPLIT;                // epilogue warps: 16 or 8
-  constexpr int CH = NCOLS / NSPLIT;            // query rows (TMEM columns) per epilogue thread: 16 or 8
+  constexpr int EW = 16;                        // epilogue warps: 8 for the first visit (sums), 8 for the second (maxima)
+  constexpr int EWV = EW / 2;                   // per visit: two warps per TMEM lane quadrant, half of the columns each
+  constexpr int CW = NCOLS / 2;                 // query rows (TMEM columns) per epilogue thread: 8, 16 or 32
+  constexpr int CHK = CW < 16 ? CW : 16;        // columns per tensor-memory load
+  constexpr int NCH = CW / CHK;                 // loads per tile and thread: 1 or 2
   constexpr int NI = NCOLS / G;          // lookahead slots per key in the running-max array
   constexpr int KSUB = D / 64;           // 64-wide sub-tiles per key tile
-  constexpr int GRP = group_tiles(D);    // key tiles per pipeline stage
-  constexpr int kStageBytes = GRP * KSUB * kSubTileBytes;
-  constexpr int kTmemCols = kTmemStages * GRP * NCOLS;
-  static_assert(CH % G == 0, "a thread must own whole GQA groups");
+  constexpr int kSlotBytes = KSUB * kSubTileBytes;          // one key tile
+  constexpr int kStageBytes = 2 * kSlotBytes;               // slot 0: first-visit tile, slot 1: second-visit tile
+  constexpr int kQSub = q_sub_tile_bytes(NCOLS);
+  constexpr int kQSlotBytes = KSUB * kQSub;
+  constexpr int kTmemCols = kTmemStages * 2 * NCOLS;
+  static_assert(CHK % G == 0, "a thread must own whole GQA groups");
 
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment by offsetting the shared array itself, so that the compiler still knows these are
@@ -362,9 +406,10 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   unsigned char* k_tiles = smem + lay.k_off;
   unsigned char* q_tiles = smem + lay.q_off;
   float* amax = reinterpret_cast<float*>(smem + lay.amax_off);       // [local tile][NI][128]
-  float* ref_slots = reinterpret_cast<float*>(smem + lay.ref_off);   // [kRefSlots][64]
+  float* xbuf = reinterpret_cast<float*>(smem + lay.xbuf_off);         // [NCOLS][128]: per-key partial row sums of one slab
+  float* ref_slots = reinterpret_cast<float*>(smem + lay.ref_off);   // [kRefSlots]: slab references, kept until the log-sum-exp warp has used them
   float* rowoff = reinterpret_cast<float*>(smem + lay.rowoff_off);   // [4 slots][64]: what the epilogue subtracts per row
-  volatile int* misc = reinterpret_cast<volatile int*>(smem + lay.misc_off);  // [0] abort, [1] tmem base, [2] is_last
+  volatile int* misc = reinterpret_cast<volatile int*>(smem + lay.misc_off);  // [0] abort, [1] tmem base, [3] references written
   const Bars bars{smem_u32(smem + lay.bar_off), a.k_stages};
   const Abort ab{misc, a.dev_status};
 
@@ -379,6 +424,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     misc[0] = 0;
     misc[1] = 0;
     misc[2] = 0;
+    misc[3] = 0;
     for (int s = 0; s < a.k_stages; ++s) {
       mbar_init(bars.k_full(s), 1);
       mbar_init(bars.k_empty(s), 1);
@@ -393,15 +439,17 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     }
     for (int x = 0; x < 4; ++x) {
       mbar_init(bars.o_ready(x), 1);
-      mbar_init(bars.o_free(x), EW);
+      mbar_init(bars.o_free(x), EWV);
     }
     mbar_init(bars.epi_sync(), EW);
     mbar_init(bars.mma_done(), kIssuers);
-    for (int b = 0; b < kPubSlots; ++b) mbar_init(bars.pub_ready(b), EW);
+    for (int b = 0; b < kPubSlots; ++b) mbar_init(bars.pub_ready(b), EWV);
+    mbar_init(bars.x_ready(), EWV);
+    mbar_init(bars.x_free(), EWV);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // zero the query stages: rows the TMA box does not cover must read as zero
-  for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kQStages * KSUB * kQSubTileBytes; i += kThreads * 16)
+  for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kQStages * 2 * kQSlotBytes; i += kThreads * 16)
     *reinterpret_cast<uint4*>(q_tiles + i) = make_uint4(0, 0, 0, 0);
   for (int i = threadIdx.x; i < my_tiles * NI * kTileKeys; i += kThreads) amax[i] = -INFINITY;
   fence_async_smem();
@@ -418,33 +466,37 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
 
   // ------------------------------------------------------------------ roles
   if (warp == 0) {
-    // ===== TMA producer: one query tile per visit, then the CTA's key tiles of the slab =====
+    // ===== TMA producer: per run t the query tiles of both slabs, then per key tile of the CTA one stage holding
+    // the tile of slab t (first visit, slot 0) and the same tile of slab t - lag (second visit, slot 1) =====
     if (lane == 0) {
       Ring kr(a.k_stages), qr(kQStages);
+      const uint64_t policy[2] = {l2_policy_keep(), l2_policy_drop()};
       bool ok = true;
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
-        for (int visit = 0; ok && visit < 2; ++visit) {
-          const int slab = visit == 0 ? t : t - a.lag;
-          if (slab < 0 || slab >= n_slabs) continue;
-          const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
-          if (!(ok = mbar_wait(bars.q_empty(qr.stage), qr.phase ^ 1u, ab))) break;
-          mbar_expect_tx(bars.q_full(qr.stage), (uint32_t)(KSUB * rows_real * 128));
+        const bool v1 = t < n_slabs, v2 = t >= a.lag;
+        const int slab_of[2] = {t, t - a.lag};
+        const bool valid[2] = {v1, v2};
+        if (!(ok = mbar_wait(bars.q_empty(qr.stage), qr.phase ^ 1u, ab))) break;
+        mbar_expect_tx(bars.q_full(qr.stage), (uint32_t)(((int)v1 + (int)v2) * KSUB * rows_real * 128));
+        for (int v = 0; v < 2; ++v) {
+          if (!valid[v]) continue;
           for (int h = 0; h < KSUB; ++h)
-            tma_load_4d(smem_u32(q_tiles + (qr.stage * KSUB + h) * kQSubTileBytes), &maps.q, h * 64, 0, 0, slab,
+            tma_load_4d(smem_u32(q_tiles + (qr.stage * 2 + v) * kQSlotBytes + h * kQSub), &maps.q, h * 64, 0, 0, slab_of[v],
                         bars.q_full(qr.stage));
-          qr.advance();
-          for (int lt0 = 0; lt0 < my_tiles; lt0 += GRP) {
-            const int n = min(GRP, my_tiles - lt0);
-            if (!(ok = mbar_wait(bars.k_empty(kr.stage), kr.phase ^ 1u, ab))) break;
-            mbar_expect_tx(bars.k_full(kr.stage), (uint32_t)(n * KSUB * kSubTileBytes));
-            for (int j = 0; j < n; ++j) {
-              const int key0 = (cta + (lt0 + j) * n_cta) * kTileKeys;
-              for (int h = 0; h < KSUB; ++h)
-                tma_load_3d(smem_u32(k_tiles + kr.stage * kStageBytes + (j * KSUB + h) * kSubTileBytes), &maps.k[layer],
-                            h * 64, key0, hk, bars.k_full(kr.stage));
-            }
-            kr.advance();
+        }
+        qr.advance();
+        for (int lt = 0; lt < my_tiles; ++lt) {
+          const int key0 = (cta + lt * n_cta) * kTileKeys;
+          if (!(ok = mbar_wait(bars.k_empty(kr.stage), kr.phase ^ 1u, ab))) break;
+          mbar_expect_tx(bars.k_full(kr.stage), (uint32_t)(((int)v1 + (int)v2) * kSlotBytes));
+          for (int v = 0; v < 2; ++v) {
+            if (!valid[v]) continue;
+            const int layer = slab_of[v] / a.n_kv_heads, hk = slab_of[v] % a.n_kv_heads;
+            for (int h = 0; h < KSUB; ++h)
+              tma_load_3d(smem_u32(k_tiles + kr.stage * kStageBytes + v * kSlotBytes + h * kSubTileBytes), &maps.k[layer],
+                          h * 64, key0, hk, bars.k_full(kr.stage), policy[v]);
           }
+          kr.advance();
         }
       }
     }
@@ -452,52 +504,45 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     // ===== MMA issuer.  The whole warp walks the loop (addresses and descriptors stay warp-uniform); one elected
     // lane issues the tensor-core instructions =====
     {
-      const int me = 0;
       Ring kr(a.k_stages), qr(kQStages), tr(kTmemStages);
       constexpr uint32_t idesc = instr_desc(NCOLS);
       const uint64_t k_desc0 = smem_desc(smem_u32(k_tiles));
       const uint64_t q_desc0 = smem_desc(smem_u32(q_tiles));
       bool ok = true;
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
-        for (int visit = 0; ok && visit < 2; ++visit) {
-          const int slab = visit == 0 ? t : t - a.lag;
-          if (slab < 0 || slab >= n_slabs) continue;
-          if (!(ok = mbar_wait_warp(bars.q_full(qr.stage), qr.phase, ab))) break;
-          const uint64_t bd0 = q_desc0 + (uint64_t)((qr.stage * KSUB * kQSubTileBytes) >> 4);
-          for (int lt0 = 0, grp = 0; lt0 < my_tiles; lt0 += GRP, ++grp) {
-            if (grp % kIssuers == me) {
-              const int n = min(GRP, my_tiles - lt0);
-              if (!(ok = mbar_wait_warp(bars.k_full(kr.stage), kr.phase, ab))) break;
-              if (!(ok = mbar_wait_warp(bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
-              tc_fence_after();
-              const uint32_t d_tmem = tmem_base + (uint32_t)(tr.stage * GRP * NCOLS);
-              const uint64_t ad0 = k_desc0 + (uint64_t)((kr.stage * kStageBytes) >> 4);
-              if (elect_one()) {
+        const bool v1 = t < n_slabs, v2 = t >= a.lag;
+        if (!(ok = mbar_wait_warp(bars.q_full(qr.stage), qr.phase, ab))) break;
+        const uint64_t bd0 = q_desc0 + (uint64_t)((qr.stage * 2 * kQSlotBytes) >> 4);
+        for (int lt = 0; lt < my_tiles; ++lt) {
+          if (!(ok = mbar_wait_warp(bars.k_full(kr.stage), kr.phase, ab))) break;
+          if (!(ok = mbar_wait_warp(bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(tr.stage * 2 * NCOLS);
+          const uint64_t ad0 = k_desc0 + (uint64_t)((kr.stage * kStageBytes) >> 4);
+          if (elect_one()) {
 #pragma unroll
-                for (int j = 0; j < GRP; ++j) {
-                  if (j < n) {
+            for (int v = 0; v < 2; ++v) {
+              if (v == 0 ? v1 : v2) {
 #pragma unroll
-                    for (int h = 0; h < KSUB; ++h) {
+                for (int h = 0; h < KSUB; ++h) {
 #pragma unroll
-                      for (int ks = 0; ks < 4; ++ks)
-                        tc_mma(d_tmem + (uint32_t)(j * NCOLS), ad0 + (uint64_t)(((j * KSUB + h) * kSubTileBytes) >> 4) + 2u * ks,
-                               bd0 + (uint64_t)((h * kQSubTileBytes) >> 4) + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
-                    }
-                  }
+                  for (int ks = 0; ks < 4; ++ks)
+                    tc_mma(d_tmem + (uint32_t)(v * NCOLS), ad0 + (uint64_t)((v * kSlotBytes + h * kSubTileBytes) >> 4) + 2u * ks,
+                           bd0 + (uint64_t)((v * kQSlotBytes + h * kQSub) >> 4) + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
                 }
-                tc_commit(bars.k_empty(kr.stage));             // one pair of commits per stage, however many tiles
-                tc_commit(bars.t_full(tr.stage));
               }
-              __syncwarp();
             }
-            kr.advance();
-            tr.advance();
+            tc_commit(bars.k_empty(kr.stage));
+            tc_commit(bars.t_full(tr.stage));
           }
-          if (!ok) break;
-          if (elect_one()) tc_commit(bars.q_empty(qr.stage));   // arrives once this warp's MMAs of the run are done
           __syncwarp();
-          qr.advance();
+          kr.advance();
+          tr.advance();
         }
+        if (!ok) break;
+        if (elect_one()) tc_commit(bars.q_empty(qr.stage));   // arrives once the MMAs of the run are done
+        __syncwarp();
+        qr.advance();
       }
       // leave only after everything issued has completed and signalled its barriers
       if (ok) {
@@ -506,214 +551,308 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         mbar_wait_warp(bars.mma_done(), 0u, ab);
       }
     }
-  } else if (warp == 3) {
-    // ===== publisher: once the epilogue warps have added their shares of a slab's row sums, order those
-    // additions before the arrival count and report this CTA (keeps the fence off the epilogue warps) =====
-    if (lane == 0) {
-      for (int slab = 0; slab < n_slabs; ++slab) {
-        if (!mbar_wait(bars.pub_ready(slab % kPubSlots), (uint32_t)(slab / kPubSlots) & 1u, ab)) break;
-        __threadfence();
-        atomicAdd(a.counters + slab, 1u);
-      }
-    }
   } else if (warp == 2) {
-    // ===== control warp: the per-row offsets the epilogue subtracts; lane handles rows lane and lane + 32 =====
+    // ===== log-sum-exp warp: once every CTA has added its share of a slab's row sums, turns the exact totals into
+    // the per-row offsets of the second visit; lane handles rows lane and lane + 32 =====
     bool ok = true;
-    const int64_t sample_key = a.n_tokens / 2;                  // the same key for every CTA: one reference per row
-    for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
-      for (int visit = 0; ok && visit < 2; ++visit) {
-        const int slab = visit == 0 ? t : t - a.lag;
-        if (slab < 0 || slab >= n_slabs) continue;
-        const int x = visit * 2 + (slab & 1);
-        const int use = slab >> 1;                              // how often step x was written before
-        float value[2] = {0.f, 0.f};                            // offsets of rows lane, lane + 32
-        if (visit == 0) {
-          // reference logit of a row: its logit against one sample key of the slab, plus a margin
-          const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
-          const uint4* krow = reinterpret_cast<const uint4*>(a.k_layers[layer] + hk * a.stride_head + sample_key * a.stride_tok);
-          const uint4* qrow[2];
+    for (int slab = 0; ok && slab < n_slabs; ++slab) {
+      const int x = 2 + (slab & 1);
+      const int use = slab >> 1;                                // how often slot x was written before
+      if (!(ok = __all_sync(0xffffffffu, count_wait(a.counters + slab, (unsigned)n_cta, ab)))) break;
+      unsigned long long w[2][kLimbs];
 #pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            const int row = min(lane + 32 * r, rows_real - 1);
-            qrow[r] = reinterpret_cast<const uint4*>(a.q + (((int64_t)slab * G + row % G) * a.n_lookahead + row / G) * D);
+      for (int r = 0; r < 2; ++r) {
+        const int row = min(lane + 32 * r, rows_real - 1);
+        const unsigned long long* acc = a.limbs + ((int64_t)slab * NCOLS + row) * kLimbStride;
+#pragma unroll
+        for (int i = 0; i < kLimbs; ++i) w[r][i] = __ldcg(acc + i);
+      }
+      // the reference of this slab was written by the reference warp at least `lag` runs ago
+      if (!(ok = __all_sync(0xffffffffu, flag_wait(&misc[3], slab + 1, ab)))) break;
+      const float ref = ref_slots[slab % kRefSlots];
+      float value[2] = {0.f, 0.f};
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int row = lane + 32 * r;
+        if (row < rows_real) {
+          double total = 0.0;                                  // sum of limb_i * 2^(40 i - 149), exact to 2^-53
+#pragma unroll
+          for (int i = kLimbs - 1; i >= 0; --i) total += __longlong_as_double((long long)(1023 + 40 * i - 149) << 52) * (double)w[r][i];
+          // log2 of the total: its binary exponent plus the log2 of its mantissa in single precision
+          const long long tb = __double_as_longlong(total);
+          const int expo = (int)((tb >> 52) & 0x7ff) - 1023;
+          const float mant = (float)__longlong_as_double((tb & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
+          float lse2 = ref + ((float)expo + log2f(mant));
+          if (!(total > 0.0) || expo == 1024) lse2 = INFINITY;  // an empty or overflowed row sum
+          if (!(lse2 > -INFINITY && lse2 < INFINITY) && a.dev_status != nullptr)
+            atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
+          value[r] = lse2 * a.inv_c;                            // lse in q.k units
+          if (cta == 0 && a.lse_out != nullptr) a.lse_out[((int64_t)slab * G + row % G) * a.n_lookahead + row / G] = lse2 * kLn2;
+        }
+      }
+      if (use > 0) {
+        if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
+      }
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int row = lane + 32 * r;
+        if (row < NCOLS) rowoff[x * 64 + row] = value[r];
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars.o_ready(x));
+    }
+  } else if (warp == 3) {
+    // ===== reference / publisher warp.  Per slab: the reference of the first visit (the largest logit of the slab's
+    // rows against one fixed sample key, plus a margin), written as soon as the slot of slab - 2 is free; then, once
+    // the shares of slab - 2 have been added to the accumulators, orders those additions before the arrival count
+    // and reports this CTA (keeps the fence off the epilogue warps) =====
+    bool ok = true;
+    const int64_t sample_key = a.n_tokens / 2;                  // the same key for every CTA: one reference per slab
+    for (int slab = 0; ok && slab < n_slabs + 2; ++slab) {
+      if (slab < n_slabs) {
+        const int x = slab & 1;
+        const int use = slab >> 1;
+        const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
+        const uint4* krow = reinterpret_cast<const uint4*>(a.k_layers[layer] + hk * a.stride_head + sample_key * a.stride_tok);
+        const uint4* qrow[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const int row = min(lane + 32 * r, rows_real - 1);
+          qrow[r] = reinterpret_cast<const uint4*>(a.q + (((int64_t)slab * G + row % G) * a.n_lookahead + row / G) * D);
+        }
+        float dot[2] = {0.f, 0.f};
+#pragma unroll
+        for (int half = 0; half < D / 64; ++half) {
+          uint4 kv[8], qv[2][8];
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch) {
+            kv[ch] = __ldg(krow + half * 8 + ch);
+            qv[0][ch] = __ldg(qrow[0] + half * 8 + ch);
+            qv[1][ch] = __ldg(qrow[1] + half * 8 + ch);
           }
-          float dot[2] = {0.f, 0.f};
 #pragma unroll
-          for (int half = 0; half < D / 64; ++half) {
-            uint4 kv[8], qv[2][8];
+          for (int ch = 0; ch < 8; ++ch) {
+            const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv[ch]);
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-              kv[ch] = __ldg(krow + half * 8 + ch);
-              qv[0][ch] = __ldg(qrow[0] + half * 8 + ch);
-              qv[1][ch] = __ldg(qrow[1] + half * 8 + ch);
-            }
+            for (int r = 0; r < 2; ++r) {
+              const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv[r][ch]);
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-              const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv[ch]);
-#pragma unroll
-              for (int r = 0; r < 2; ++r) {
-                const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv[r][ch]);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  const float2 kf = __bfloat1622float2(k2[e]), qf = __bfloat1622float2(q2[e]);
-                  dot[r] = fmaf(kf.x, qf.x, fmaf(kf.y, qf.y, dot[r]));
-                }
+              for (int e = 0; e < 4; ++e) {
+                const float2 kf = __bfloat1622float2(k2[e]), qf = __bfloat1622float2(q2[e]);
+                dot[r] = fmaf(kf.x, qf.x, fmaf(kf.y, qf.y, dot[r]));
               }
             }
           }
-#pragma unroll
-          for (int r = 0; r < 2; ++r)
-            if (lane + 32 * r < rows_real) value[r] = fmaf(dot[r], a.c, kRefMargin);   // reference, base-2 units
-        } else {
-          // all shares of the slab's row sums are in once every CTA has reported
-          if (!(ok = __all_sync(0xffffffffu, count_wait(a.counters + slab, (unsigned)n_cta, ab)))) break;
-#pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            const int row = lane + 32 * r;
-            if (row < rows_real) {
-              const unsigned long long* acc = a.limbs + ((int64_t)slab * NCOLS + row) * kLimbStride;
-              unsigned long long w[kLimbs];
-#pragma unroll
-              for (int i = 0; i < kLimbs; ++i) w[i] = __ldcg(acc + i);
-              double total = 0.0;                              // sum of limb_i * 2^(40 i - 149), exact to 2^-53
-#pragma unroll
-              for (int i = kLimbs - 1; i >= 0; --i) total += __longlong_as_double((long long)(1023 + 40 * i - 149) << 52) * (double)w[i];
-              const float lse2 = ref_slots[(slab % kRefSlots) * 64 + row] + (float)log2(total);
-              if (!(lse2 > -INFINITY && lse2 < INFINITY) && a.dev_status != nullptr)
-                atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
-              value[r] = lse2 * a.inv_c;                          // lse in q.k units
-              if (cta == 0 && a.lse_out != nullptr) a.lse_out[((int64_t)slab * G + row % G) * a.n_lookahead + row / G] = lse2 * kLn2;
-            }
-          }
         }
+        // one reference per slab: the largest sample logit of its rows (padding rows repeat a real one), base-2 units
+        float ref = fmaxf(dot[0], dot[1]);
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) ref = fmaxf(ref, __shfl_xor_sync(0xffffffffu, ref, off));
+        ref = fmaf(ref, a.c, kRefMargin);
         if (use > 0) {
           if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
         }
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          const int row = lane + 32 * r;
-          if (row < NCOLS) {
-            rowoff[x * 64 + row] = value[r];
-            if (visit == 0) ref_slots[(slab % kRefSlots) * 64 + row] = value[r];
-          }
+        if (lane == 0) {
+          rowoff[x * 64] = ref;
+          ref_slots[slab % kRefSlots] = ref;
+          __threadfence_block();
+          misc[3] = slab + 1;                                    // the log-sum-exp warp reads ref_slots after this
+          mbar_arrive(bars.o_ready(x));
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars.o_ready(x));
+      }
+      if (slab >= 2) {
+        const int ps = slab - 2;
+        if (!(ok = mbar_wait_warp(bars.pub_ready(ps % kPubSlots), (uint32_t)(ps / kPubSlots) & 1u, ab))) break;
+        if (lane == 0) {
+          __threadfence();
+          atomicAdd(a.counters + ps, 1u);
+        }
+        __syncwarp();
       }
     }
   } else if (warp >= 4 && warp < 4 + EW) {
-    // ===== epilogue: EW warps; warp % 4 picks the TMEM lane quadrant (32 keys), (warp - 4) / 4 the slice of CH columns.
-    // With 64 query rows four warps share a quadrant: they hide each other's barrier and TMEM-load latencies =====
+    // ===== epilogue.  Warps 4..11 ("sum" warps) take the first-visit tile of every stage, warps 12..19 ("max" warps)
+    // the second-visit tile; warp % 4 picks the TMEM lane quadrant (32 keys), the next bit the half of the query
+    // rows.  The two groups run on their own: the exp2-bound and the max-bound work overlap on each scheduler, and
+    // a tensor-memory load of one chunk is in flight while the previous chunk is processed =====
     const int quad = warp & 3;
-    const int hh = (warp - 4) >> 2;
+    const bool is_sum = warp < 4 + EWV;
+    const int half = ((warp - 4) >> 2) & 1;
     const int et = threadIdx.x - 128;                           // index among the epilogue threads
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const int n_full_tiles = (int)(a.n_tokens / kTileKeys);     // tiles below this index have 128 real keys
     Ring tr(kTmemStages);
     EpiSync es{bars.epi_sync()};
     bool ok = true;
-    for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
-      for (int visit = 0; ok && visit < 2; ++visit) {
-        const int slab = visit == 0 ? t : t - a.lag;
-        if (slab < 0 || slab >= n_slabs) continue;
-        // this run's row offsets (reference or lse) of the thread's columns
-        const int x = visit * 2 + (slab & 1);
-        if (!(ok = mbar_wait_warp(bars.o_ready(x), (uint32_t)(slab >> 1) & 1u, ab))) break;
-        float off[CH];
-#pragma unroll
-        for (int j = 0; j < CH; ++j) off[j] = rowoff[x * 64 + hh * CH + j];
+    if (is_sum) {
+      for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
+        if (t >= n_slabs) {
+          // nothing to sum any more: keep the stage hand-over going
+          for (int lt = 0; lt < my_tiles; ++lt) {
+            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+            if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
+            tr.advance();
+          }
+          continue;
+        }
+        const int slab = t, x1 = slab & 1;
+        if (!(ok = mbar_wait_warp(bars.o_ready(x1), (uint32_t)(slab >> 1) & 1u, ab))) break;
+        const float nref = -rowoff[x1 * 64];                    // one reference per slab
         __syncwarp();
-        if (lane == 0) mbar_arrive(bars.o_free(x));
-        // tile loop shared by both visits
-        float sum[CH];
+        if (lane == 0) mbar_arrive(bars.o_free(x1));
+        float sum[CW];
 #pragma unroll
-        for (int j = 0; j < CH; ++j) sum[j] = 0.f;
-        auto process = [&](const uint32_t (&r)[CH], int lt) {
-          if (visit == 0) {
-            // visit 1: per-thread sums of exp2 over the thread's keys
-            const int64_t key = (int64_t)(cta + lt * n_cta) * kTileKeys + quad * 32 + lane;
-            if (key < a.n_tokens) {
-#pragma unroll
-              for (int j = 0; j < CH; ++j) sum[j] += fast_exp2(fmaf(__uint_as_float(r[j]), a.c, -off[j]));
-            }
-          } else {
-            // visit 2: running max over (layer, head) of q.k - lse/c
-            float* slot = amax + ((int64_t)lt * NI + hh * (CH / G)) * kTileKeys + quad * 32 + lane;
-#pragma unroll
-            for (int ii = 0; ii < CH / G; ++ii) {
-              float mx = __uint_as_float(r[ii * G]) - off[ii * G];
-#pragma unroll
-              for (int g = 1; g < G; ++g) mx = fmaxf(mx, __uint_as_float(r[ii * G + g]) - off[ii * G + g]);
-              if (hh * (CH / G) + ii < a.n_lookahead) slot[ii * kTileKeys] = fmaxf(slot[ii * kTileKeys], mx);
-            }
+        for (int j = 0; j < CW; ++j) sum[j] = 0.f;
+        uint32_t rb[2][CHK];
+        bool pending = false;                                   // chunk 0 of the current stage is already on its way
+        for (int lt = 0; lt < my_tiles; ++lt) {
+          const int tile = cta + lt * n_cta;
+          const bool real = tile < n_full_tiles || (int64_t)tile * kTileKeys + quad * 32 + lane < a.n_tokens;
+          const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(tr.stage * 2 * NCOLS + half * CW);
+          if (!pending) {
+            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+            tc_fence_after();
+            tmem_issue<CHK>(taddr, rb[0]);
           }
-        };
-        for (int lt0 = 0; lt0 < my_tiles; lt0 += GRP) {
-          const int n = min(GRP, my_tiles - lt0);
-          if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
-          tc_fence_after();
-          const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(tr.stage * GRP * NCOLS + hh * CH);
+          pending = false;
 #pragma unroll
-          for (int j = 0; j < GRP; ++j) {
-            if (j < n) {
-              uint32_t r[CH];
-              tmem_issue<CH>(taddr + (uint32_t)(j * NCOLS), r);
-              tmem_wait<CH>(r);
-              if (j == n - 1) {
-                // the stage can be overwritten: its last tile is in registers
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
+          for (int c = 0; c < NCH; ++c) {
+            tmem_wait<CHK>(rb[c & 1]);
+            if (c + 1 < NCH) {
+              tmem_issue<CHK>(taddr + (uint32_t)((c + 1) * CHK), rb[(c + 1) & 1]);
+            } else {
+              // the stage can be overwritten: its last chunk is in registers
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
+              tr.advance();
+              if (NCH == 2 && lt + 1 < my_tiles) {
+                if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+                tc_fence_after();
+                tmem_issue<CHK>(tmem_base + lane_addr + (uint32_t)(tr.stage * 2 * NCOLS + half * CW), rb[(c + 1) & 1]);
+                pending = true;
               }
-              process(r, lt0 + j);
+            }
+            // per-thread sums of exp2 over the thread's keys
+            if (real) {
+#pragma unroll
+              for (int j = 0; j < CHK; ++j) sum[c * CHK + j] += fast_exp2(fmaf(__uint_as_float(rb[c & 1][j]), a.c, nref));
             }
           }
-          tr.advance();
+          if (!ok) break;
         }
         if (!ok) break;
-        if (visit == 0) {
-          // reduce over the 32 keys of the warp: transposing butterfly while more than one column is
-          // left per thread, plain butterfly afterwards
-          {
-            int width = CH;
+        // hand the per-key sums to the max warps through shared memory: they have the slack to add them up over
+        // the 128 keys and into the row accumulators (in a fixed order, so the result stays deterministic)
+        if (slab > 0) {
+          if (!(ok = mbar_wait_warp(bars.x_free(), (uint32_t)(slab - 1) & 1u, ab))) break;
+        }
 #pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) {
-              if (width > 1) {
-                width >>= 1;
-                const bool upper = (lane & off) != 0;
+        for (int j = 0; j < CW; ++j) xbuf[(half * CW + j) * kTileKeys + quad * 32 + lane] = sum[j];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars.x_ready());
+      }
+    } else {
+      // adds up the per-key sums of slab `slab` (written by the sum warps) and adds each row's total, exactly, to the
+      // row's fixed-point accumulator (value = mantissa * 2^(p - 149), p = biased exponent - 1)
+      constexpr int XC = NCOLS / EWV;                          // rows per max warp: 2, 4 or 8
+      const int xw = warp - 4 - EWV;                           // 0..7
+      auto reduce_slab = [&](int slab) -> bool {
+        if (!mbar_wait_warp(bars.x_ready(), (uint32_t)slab & 1u, ab)) return false;
+        float tot = 0.f;
 #pragma unroll
-                for (int j = 0; j < CH / 2; ++j) {
-                  if (j < width) {
-                    const float send = upper ? sum[j] : sum[j + width];
-                    const float keep = upper ? sum[j + width] : sum[j];
-                    sum[j] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-                  }
-                }
-              } else {
-                sum[0] += __shfl_xor_sync(0xffffffffu, sum[0], off);
+        for (int j = 0; j < XC; ++j) {
+          const float4 v = *reinterpret_cast<const float4*>(xbuf + (xw * XC + j) * kTileKeys + lane * 4);
+          float sacc = (v.x + v.y) + (v.z + v.w);
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, off);
+          if (lane == j) tot = sacc;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars.x_free());
+        if (lane < XC) {
+          const uint32_t bits = __float_as_uint(tot);
+          const uint32_t expo = bits >> 23;                  // sums are non-negative: no sign bit
+          if (expo == 255u) {
+            if (a.dev_status != nullptr) atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
+          } else if (expo != 0u) {
+            const unsigned long long mant = (unsigned long long)((bits & 0x7FFFFFu) | 0x800000u);
+            const uint32_t pos = expo - 1u, limb = pos / 40u, off = pos % 40u;
+            unsigned long long* acc = a.limbs + ((int64_t)slab * NCOLS + xw * XC + lane) * kLimbStride + limb;
+            const unsigned long long lo = (mant << off) & ((1ull << 40) - 1ull), hi = mant >> (40u - off);
+            atomicAdd(acc, lo);
+            if (hi != 0ull) atomicAdd(acc + 1, hi);
+          }
+        }
+        // hand over to the publisher warp, which makes the additions visible and counts this CTA in
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars.pub_ready(slab % kPubSlots));
+        return true;
+      };
+      for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
+        if (t < a.lag) {
+          for (int lt = 0; lt < my_tiles; ++lt) {
+            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+            if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
+            tr.advance();
+          }
+          if (ok && t < n_slabs) ok = reduce_slab(t);
+          continue;
+        }
+        const int slab = t - a.lag, x2 = 2 + (slab & 1);
+        if (!(ok = mbar_wait_warp(bars.o_ready(x2), (uint32_t)(slab >> 1) & 1u, ab))) break;
+        const float4* off2 = reinterpret_cast<const float4*>(rowoff + x2 * 64 + half * CW);
+        uint32_t rb[2][CHK];
+        bool pending = false;
+        for (int lt = 0; lt < my_tiles; ++lt) {
+          const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(tr.stage * 2 * NCOLS + NCOLS + half * CW);
+          if (!pending) {
+            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+            tc_fence_after();
+            tmem_issue<CHK>(taddr, rb[0]);
+          }
+          pending = false;
+          float* slot = amax + ((int64_t)lt * NI + half * (CW / G)) * kTileKeys + quad * 32 + lane;
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) {
+            tmem_wait<CHK>(rb[c & 1]);
+            if (c + 1 < NCH) {
+              tmem_issue<CHK>(taddr + (uint32_t)((c + 1) * CHK), rb[(c + 1) & 1]);
+            } else {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
+              tr.advance();
+              if (NCH == 2 && lt + 1 < my_tiles) {
+                if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+                tc_fence_after();
+                tmem_issue<CHK>(tmem_base + lane_addr + (uint32_t)(tr.stage * 2 * NCOLS + NCOLS + half * CW), rb[(c + 1) & 1]);
+                pending = true;
               }
             }
-          }
-          // the lane now holds the warp total of column hh * CH + lane / (32 / CH): add it, exactly, to the
-          // row's fixed-point accumulator (value = mantissa * 2^(p - 149), p = biased exponent - 1)
-          constexpr int kLanesPerCol = 32 / CH;
-          if (lane % kLanesPerCol == 0) {
-            const uint32_t bits = __float_as_uint(sum[0]);
-            const uint32_t expo = bits >> 23;                  // sums are non-negative: no sign bit
-            if (expo == 255u) {
-              if (a.dev_status != nullptr) atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
-            } else if (expo != 0u) {
-              const unsigned long long mant = (unsigned long long)((bits & 0x7FFFFFu) | 0x800000u);
-              const uint32_t pos = expo - 1u, limb = pos / 40u, off = pos % 40u;
-              unsigned long long* acc = a.limbs + ((int64_t)slab * NCOLS + hh * CH + lane / kLanesPerCol) * kLimbStride + limb;
-              const unsigned long long lo = (mant << off) & ((1ull << 40) - 1ull), hi = mant >> (40u - off);
-              atomicAdd(acc, lo);
-              if (hi != 0ull) atomicAdd(acc + 1, hi);
+            float o[CHK];
+#pragma unroll
+            for (int j = 0; j < CHK / 4; ++j) {
+              const float4 v = off2[c * (CHK / 4) + j];
+              o[4 * j] = v.x; o[4 * j + 1] = v.y; o[4 * j + 2] = v.z; o[4 * j + 3] = v.w;
+            }
+            // running max over (layer, head) of q.k - lse/c
+#pragma unroll
+            for (int ii = 0; ii < CHK / G; ++ii) {
+              float mx = __uint_as_float(rb[c & 1][ii * G]) - o[ii * G];
+#pragma unroll
+              for (int g = 1; g < G; ++g) mx = fmaxf(mx, __uint_as_float(rb[c & 1][ii * G + g]) - o[ii * G + g]);
+              const int i = c * (CHK / G) + ii;
+              if (half * (CW / G) + i < a.n_lookahead) slot[i * kTileKeys] = fmaxf(slot[i * kTileKeys], mx);
             }
           }
-          // hand over to the publisher warp, which makes the additions visible and counts this CTA in
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bars.pub_ready(slab % kPubSlots));
+          if (!ok) break;
         }
+        if (!ok) break;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars.o_free(x2));
+        if (t < n_slabs) ok = reduce_slab(t);
       }
     }
     // ---------------- importance: mean over lookahead of exp2(c * running max) ----------------
@@ -803,7 +942,7 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
 // environment variable SPF_FUSED_LAG (1..8) overrides the choice for tuning.
 int fused_lag(const ScoreProblem& p, int n_slabs) {
   const double slab_bytes = (double)p.n_tokens * p.head_dim * 2.0;
-  int lag = (int)(40.0 * 1024 * 1024 / slab_bytes) - 1;
+  int lag = (int)(80.0 * 1024 * 1024 / slab_bytes) - 1;
   lag = std::max(2, std::min(lag, 8));
   if (const char* env = getenv("SPF_FUSED_LAG")) {
     const int v = atoi(env);

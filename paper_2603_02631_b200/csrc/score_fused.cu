@@ -674,8 +674,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   } else if (warp >= 4 && warp < 4 + EW) {
     // ===== epilogue.  Warps 4..11 ("sum" warps) take the first-visit tile of every stage, warps 12..19 ("max" warps)
     // the second-visit tile; warp % 4 picks the TMEM lane quadrant (32 keys), the next bit the half of the query
-    // rows.  The two groups run on their own: the exp2-bound and the max-bound work overlap on each scheduler, and
-    // a tensor-memory load of one chunk is in flight while the previous chunk is processed =====
+    // rows.  The two groups run on their own: the exp2-bound and the max-bound work overlap on each scheduler =====
     const int quad = warp & 3;
     const bool is_sum = warp < 4 + EWV;
     const int half = ((warp - 4) >> 2) & 1;
@@ -704,43 +703,32 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         float sum[CW];
 #pragma unroll
         for (int j = 0; j < CW; ++j) sum[j] = 0.f;
-        uint32_t rb[2][CHK];
-        bool pending = false;                                   // chunk 0 of the current stage is already on its way
         for (int lt = 0; lt < my_tiles; ++lt) {
           const int tile = cta + lt * n_cta;
           const bool real = tile < n_full_tiles || (int64_t)tile * kTileKeys + quad * 32 + lane < a.n_tokens;
+          if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+          tc_fence_after();
           const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(tr.stage * 2 * NCOLS + half * CW);
-          if (!pending) {
-            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
-            tc_fence_after();
-            tmem_issue<CHK>(taddr, rb[0]);
-          }
-          pending = false;
+          // chunk by chunk: load, wait, compute.  No load is kept in flight across the arithmetic: with one pending,
+          // the warp's exp2 stream ran markedly slower (measured), and the other warps hide the latency anyway
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
-            tmem_wait<CHK>(rb[c & 1]);
-            if (c + 1 < NCH) {
-              tmem_issue<CHK>(taddr + (uint32_t)((c + 1) * CHK), rb[(c + 1) & 1]);
-            } else {
+            uint32_t r[CHK];
+            tmem_issue<CHK>(taddr + (uint32_t)(c * CHK), r);
+            tmem_wait<CHK>(r);
+            if (c + 1 == NCH) {
               // the stage can be overwritten: its last chunk is in registers
               tc_fence_before();
               __syncwarp();
               if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
               tr.advance();
-              if (NCH == 2 && lt + 1 < my_tiles) {
-                if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
-                tc_fence_after();
-                tmem_issue<CHK>(tmem_base + lane_addr + (uint32_t)(tr.stage * 2 * NCOLS + half * CW), rb[(c + 1) & 1]);
-                pending = true;
-              }
             }
             // per-thread sums of exp2 over the thread's keys
             if (real) {
 #pragma unroll
-              for (int j = 0; j < CHK; ++j) sum[c * CHK + j] += fast_exp2(fmaf(__uint_as_float(rb[c & 1][j]), a.c, nref));
+              for (int j = 0; j < CHK; ++j) sum[c * CHK + j] += fast_exp2(fmaf(__uint_as_float(r[j]), a.c, nref));
             }
           }
-          if (!ok) break;
         }
         if (!ok) break;
         // hand the per-key sums to the max warps through shared memory: they have the slack to add them up over
@@ -803,33 +791,21 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         const int slab = t - a.lag, x2 = 2 + (slab & 1);
         if (!(ok = mbar_wait_warp(bars.o_ready(x2), (uint32_t)(slab >> 1) & 1u, ab))) break;
         const float4* off2 = reinterpret_cast<const float4*>(rowoff + x2 * 64 + half * CW);
-        uint32_t rb[2][CHK];
-        bool pending = false;
         for (int lt = 0; lt < my_tiles; ++lt) {
+          if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
+          tc_fence_after();
           const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(tr.stage * 2 * NCOLS + NCOLS + half * CW);
-          if (!pending) {
-            if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
-            tc_fence_after();
-            tmem_issue<CHK>(taddr, rb[0]);
-          }
-          pending = false;
           float* slot = amax + ((int64_t)lt * NI + half * (CW / G)) * kTileKeys + quad * 32 + lane;
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
-            tmem_wait<CHK>(rb[c & 1]);
-            if (c + 1 < NCH) {
-              tmem_issue<CHK>(taddr + (uint32_t)((c + 1) * CHK), rb[(c + 1) & 1]);
-            } else {
+            uint32_t r[CHK];
+            tmem_issue<CHK>(taddr + (uint32_t)(c * CHK), r);
+            tmem_wait<CHK>(r);
+            if (c + 1 == NCH) {
               tc_fence_before();
               __syncwarp();
               if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
               tr.advance();
-              if (NCH == 2 && lt + 1 < my_tiles) {
-                if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
-                tc_fence_after();
-                tmem_issue<CHK>(tmem_base + lane_addr + (uint32_t)(tr.stage * 2 * NCOLS + NCOLS + half * CW), rb[(c + 1) & 1]);
-                pending = true;
-              }
             }
             float o[CHK];
 #pragma unroll
@@ -840,14 +816,13 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
             // running max over (layer, head) of q.k - lse/c
 #pragma unroll
             for (int ii = 0; ii < CHK / G; ++ii) {
-              float mx = __uint_as_float(rb[c & 1][ii * G]) - o[ii * G];
+              float mx = __uint_as_float(r[ii * G]) - o[ii * G];
 #pragma unroll
-              for (int g = 1; g < G; ++g) mx = fmaxf(mx, __uint_as_float(rb[c & 1][ii * G + g]) - o[ii * G + g]);
+              for (int g = 1; g < G; ++g) mx = fmaxf(mx, __uint_as_float(r[ii * G + g]) - o[ii * G + g]);
               const int i = c * (CHK / G) + ii;
               if (half * (CW / G) + i < a.n_lookahead) slot[i * kTileKeys] = fmaxf(slot[i * kTileKeys], mx);
             }
           }
-          if (!ok) break;
         }
         if (!ok) break;
         __syncwarp();

@@ -325,7 +325,7 @@ __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, i
   s.k_off = o;        o += (uint32_t)k_stages * 2 * (d / 64) * kSubTileBytes;
   s.q_off = o;        o += (uint32_t)kQStages * 2 * (d / 64) * q_sub_tile_bytes(ncols);
   s.amax_off = o;     o += (uint32_t)tiles_per_cta_max * (ncols / group) * kTileKeys * 4;
-  s.xbuf_off = o;     o += (uint32_t)ncols * kTileKeys * 4;
+  s.xbuf_off = o;     o += (uint32_t)ncols * (kTileKeys / 4) * 4;
   s.ref_off = o;      o += kRefSlots * 4;
   s.rowoff_off = o;   o += 4 * 64 * 4;
   s.bar_off = o;      o += 64 * 8;
@@ -406,7 +406,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   unsigned char* k_tiles = smem + lay.k_off;
   unsigned char* q_tiles = smem + lay.q_off;
   float* amax = reinterpret_cast<float*>(smem + lay.amax_off);       // [local tile][NI][128]
-  float* xbuf = reinterpret_cast<float*>(smem + lay.xbuf_off);         // [NCOLS][128]: per-key partial row sums of one slab
+  float* xbuf = reinterpret_cast<float*>(smem + lay.xbuf_off);         // [NCOLS][32]: partial row sums of one slab, each over four keys
   float* ref_slots = reinterpret_cast<float*>(smem + lay.ref_off);   // [kRefSlots]: slab references, kept until the log-sum-exp warp has used them
   float* rowoff = reinterpret_cast<float*>(smem + lay.rowoff_off);   // [4 slots][64]: what the epilogue subtracts per row
   volatile int* misc = reinterpret_cast<volatile int*>(smem + lay.misc_off);  // [0] abort, [1] tmem base, [3] references written
@@ -736,8 +736,32 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         if (slab > 0) {
           if (!(ok = mbar_wait_warp(bars.x_free(), (uint32_t)(slab - 1) & 1u, ab))) break;
         }
+        // two transposing butterfly steps first (sums over 4 keys, a quarter of the columns left per thread): the buffer
+        // is a quarter of the size, which buys another stage of the key ring
+        {
+          int width = CW;
 #pragma unroll
-        for (int j = 0; j < CW; ++j) xbuf[(half * CW + j) * kTileKeys + quad * 32 + lane] = sum[j];
+          for (int off = 16; off >= 8; off >>= 1) {
+            width >>= 1;
+            const bool upper = (lane & off) != 0;
+#pragma unroll
+            for (int j = 0; j < CW / 2; ++j) {
+              if (j < width) {
+                const float send = upper ? sum[j] : sum[j + width];
+                const float keep = upper ? sum[j + width] : sum[j];
+                sum[j] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+              }
+            }
+          }
+        }
+        {
+          const int col0 = half * CW + ((lane & 16) ? CW / 2 : 0) + ((lane & 8) ? CW / 4 : 0);
+          // the position within the row is permuted by the (lane & 24) bits so that the four column groups of a warp
+          // do not collide on the same banks; the readers add up whole rows, so the order does not matter to them
+          const int pos = ((quad ^ (lane >> 3)) & 3) * 8 + (lane & 7);
+#pragma unroll
+          for (int j = 0; j < CW / 4; ++j) xbuf[(col0 + j) * (kTileKeys / 4) + pos] = sum[j];
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars.x_ready());
       }
@@ -751,8 +775,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         float tot = 0.f;
 #pragma unroll
         for (int j = 0; j < XC; ++j) {
-          const float4 v = *reinterpret_cast<const float4*>(xbuf + (xw * XC + j) * kTileKeys + lane * 4);
-          float sacc = (v.x + v.y) + (v.z + v.w);
+          float sacc = xbuf[(xw * XC + j) * (kTileKeys / 4) + lane];
 #pragma unroll
           for (int off = 16; off >= 1; off >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, off);
           if (lane == j) tot = sacc;

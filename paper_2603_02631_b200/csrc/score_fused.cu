@@ -10,8 +10,8 @@
 // tile j of slab t - lag for visit 2 (read again by the same CTA, so from L2, with an evict-first hint).
 //
 // Work split.  The grid is persistent (one CTA per SM).  CTA b owns key tiles b, b + grid, ... (128
-// keys each) of EVERY slab, so its running maxima for those keys stay in its shared memory for the
-// whole kernel and the importance of a key is written exactly once, at the end.
+// keys each) of EVERY slab, so its running maxima for those keys stay on its SM (in tensor memory, next to
+// the accumulator stages) for the whole kernel and the importance of a key is written exactly once, at the end.
 //
 // One tile = one tcgen05 MMA group: A = 128 keys x d (shared memory, TMA, 128-byte swizzle),
 // B = the slab's query rows x d (row j = i * G + g: lookahead i, head g of the GQA group), D = fp32
@@ -58,7 +58,8 @@ constexpr int kIssuers = 1;            // MMA-issuing warps: local tile lt belon
 constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accumulators (covers every finite fp32)
 constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
 constexpr int kQStages = 2;
-constexpr int kTmemStages = 4;
+constexpr int kTmemStages = 4;         // upper bound; the launch picks 2..4 (FusedArgs::t_stages)
+constexpr int kTmemColsAll = 512;      // the CTA takes all of its SM's tensor memory
 constexpr int kRefSlots = 16;         // row references stay readable for this many slabs (must exceed the lag)
 constexpr int kPubSlots = 16;        // slabs whose hand-over to the publisher may be pending at once
 constexpr float kRefMargin = 60.f;     // base-2 units added to the sampled reference logit
@@ -74,7 +75,7 @@ struct FusedArgs {
   const __nv_bfloat16* k_layers[kFusedMaxLayers];
   const __nv_bfloat16* q;
   int64_t n_tokens, stride_head, stride_tok;
-  int n_layers, n_kv_heads, n_lookahead, n_tiles, tiles_per_cta_max, lag, k_stages;
+  int n_layers, n_kv_heads, n_lookahead, n_tiles, tiles_per_cta_max, lag, k_stages, t_stages;
   float c, inv_c;
   unsigned long long* limbs;  // [slab][NCOLS][kLimbStride] exact fixed-point sums of exp2(c*q.k - ref) over all keys
   unsigned* counters;     // [slab] CTAs whose share of the slab's row sums is in the accumulators
@@ -262,6 +263,56 @@ template <int N>
 __device__ __forceinline__ void tmem_wait(uint32_t (&r)[N]);
 
 template <>
+__device__ __forceinline__ void tmem_issue<1>(uint32_t taddr, uint32_t (&r)[1]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r[0]) : "r"(taddr));
+}
+template <>
+__device__ __forceinline__ void tmem_wait<1>(uint32_t (&r)[1]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(r[0]) : : "memory");
+}
+template <>
+__device__ __forceinline__ void tmem_issue<2>(uint32_t taddr, uint32_t (&r)[2]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(taddr));
+}
+template <>
+__device__ __forceinline__ void tmem_wait<2>(uint32_t (&r)[2]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(r[0]), "+r"(r[1]) : : "memory");
+}
+template <>
+__device__ __forceinline__ void tmem_issue<4>(uint32_t taddr, uint32_t (&r)[4]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(taddr));
+}
+template <>
+__device__ __forceinline__ void tmem_wait<4>(uint32_t (&r)[4]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]) : : "memory");
+}
+// registers -> TMEM (the warp's 32 lanes, N consecutive columns); tmem_store_wait completes the thread's stores
+template <int N>
+__device__ __forceinline__ void tmem_store(uint32_t taddr, const uint32_t (&r)[N]);
+template <>
+__device__ __forceinline__ void tmem_store<1>(uint32_t taddr, const uint32_t (&r)[1]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(taddr), "r"(r[0]) : "memory");
+}
+template <>
+__device__ __forceinline__ void tmem_store<2>(uint32_t taddr, const uint32_t (&r)[2]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1,%2};" ::"r"(taddr), "r"(r[0]), "r"(r[1]) : "memory");
+}
+template <>
+__device__ __forceinline__ void tmem_store<4>(uint32_t taddr, const uint32_t (&r)[4]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};" ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3])
+               : "memory");
+}
+template <>
+__device__ __forceinline__ void tmem_store<8>(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
+               "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_store_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+template <>
 __device__ __forceinline__ void tmem_issue<8>(uint32_t taddr, uint32_t (&r)[8]) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
@@ -316,7 +367,7 @@ __device__ __forceinline__ void tmem_wait<32>(uint32_t (&r)[32]) {
 __host__ __device__ constexpr int q_sub_tile_bytes(int ncols) { return ncols * 128; }   // ncols query rows x 64 bf16
 
 struct SmemLayout {
-  uint32_t k_off, q_off, amax_off, xbuf_off, ref_off, rowoff_off, bar_off, misc_off, total;
+  uint32_t k_off, q_off, xbuf_off, ref_off, rowoff_off, bar_off, misc_off, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, int k_stages, int tiles_per_cta_max) {
@@ -324,7 +375,6 @@ __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, i
   uint32_t o = 0;
   s.k_off = o;        o += (uint32_t)k_stages * 2 * (d / 64) * kSubTileBytes;
   s.q_off = o;        o += (uint32_t)kQStages * 2 * (d / 64) * q_sub_tile_bytes(ncols);
-  s.amax_off = o;     o += (uint32_t)tiles_per_cta_max * (ncols / group) * kTileKeys * 4;
   s.xbuf_off = o;     o += (uint32_t)ncols * (kTileKeys / 4) * 4;
   s.ref_off = o;      o += kRefSlots * 4;
   s.rowoff_off = o;   o += 4 * 64 * 4;
@@ -395,7 +445,12 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   constexpr int kStageBytes = 2 * kSlotBytes;               // slot 0: first-visit tile, slot 1: second-visit tile
   constexpr int kQSub = q_sub_tile_bytes(NCOLS);
   constexpr int kQSlotBytes = KSUB * kQSub;
-  constexpr int kTmemCols = kTmemStages * 2 * NCOLS;
+  constexpr int kTmemCols = kTmemColsAll;
+  constexpr int NIH = (NCOLS / 2) / G;   // lookahead slots per max-warp thread
+  constexpr int AC = NIH < 8 ? NIH : 8;  // running maxima moved per tensor-memory load / store
+  // tensor memory: t_stages stages of 2 x NCOLS accumulator columns, then the running maxima, [local tile][NI]
+  // columns (lane = key), which therefore never leave the SM either
+  const uint32_t amax_col0 = (uint32_t)(a.t_stages * 2 * NCOLS);
   static_assert(CHK % G == 0, "a thread must own whole GQA groups");
 
   extern __shared__ unsigned char smem_raw[];
@@ -405,7 +460,6 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   const SmemLayout lay = smem_layout(D, NCOLS, G, a.k_stages, a.tiles_per_cta_max);
   unsigned char* k_tiles = smem + lay.k_off;
   unsigned char* q_tiles = smem + lay.q_off;
-  float* amax = reinterpret_cast<float*>(smem + lay.amax_off);       // [local tile][NI][128]
   float* xbuf = reinterpret_cast<float*>(smem + lay.xbuf_off);         // [NCOLS][32]: partial row sums of one slab, each over four keys
   float* ref_slots = reinterpret_cast<float*>(smem + lay.ref_off);   // [kRefSlots]: slab references, kept until the log-sum-exp warp has used them
   float* rowoff = reinterpret_cast<float*>(smem + lay.rowoff_off);   // [4 slots][64]: what the epilogue subtracts per row
@@ -433,7 +487,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       mbar_init(bars.q_full(s), 1);
       mbar_init(bars.q_empty(s), kIssuers);
     }
-    for (int s = 0; s < kTmemStages; ++s) {
+    for (int s = 0; s < a.t_stages; ++s) {
       mbar_init(bars.t_full(s), 1);
       mbar_init(bars.t_empty(s), EW);
     }
@@ -451,7 +505,6 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   // zero the query stages: rows the TMA box does not cover must read as zero
   for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kQStages * 2 * kQSlotBytes; i += kThreads * 16)
     *reinterpret_cast<uint4*>(q_tiles + i) = make_uint4(0, 0, 0, 0);
-  for (int i = threadIdx.x; i < my_tiles * NI * kTileKeys; i += kThreads) amax[i] = -INFINITY;
   fence_async_smem();
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)&misc[1])),
@@ -504,7 +557,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     // ===== MMA issuer.  The whole warp walks the loop (addresses and descriptors stay warp-uniform); one elected
     // lane issues the tensor-core instructions =====
     {
-      Ring kr(a.k_stages), qr(kQStages), tr(kTmemStages);
+      Ring kr(a.k_stages), qr(kQStages), tr(a.t_stages);
       constexpr uint32_t idesc = instr_desc(NCOLS);
       const uint64_t k_desc0 = smem_desc(smem_u32(k_tiles));
       const uint64_t q_desc0 = smem_desc(smem_u32(q_tiles));
@@ -678,10 +731,9 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     const int quad = warp & 3;
     const bool is_sum = warp < 4 + EWV;
     const int half = ((warp - 4) >> 2) & 1;
-    const int et = threadIdx.x - 128;                           // index among the epilogue threads
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const int n_full_tiles = (int)(a.n_tokens / kTileKeys);     // tiles below this index have 128 real keys
-    Ring tr(kTmemStages);
+    Ring tr(a.t_stages);
     EpiSync es{bars.epi_sync()};
     bool ok = true;
     if (is_sum) {
@@ -801,6 +853,16 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         if (lane == 0) mbar_arrive(bars.pub_ready(slab % kPubSlots));
         return true;
       };
+      {
+        uint32_t ninf[AC];
+#pragma unroll
+        for (int j = 0; j < AC; ++j) ninf[j] = 0xff800000u;      // -inf
+        for (int lt = 0; lt < my_tiles; ++lt)
+#pragma unroll
+          for (int q = 0; q < NIH / AC; ++q)
+            tmem_store<AC>(tmem_base + lane_addr + amax_col0 + (uint32_t)(lt * NI + half * NIH + q * AC), ninf);
+        tmem_store_wait();
+      }
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
         if (t < a.lag) {
           for (int lt = 0; lt < my_tiles; ++lt) {
@@ -818,12 +880,20 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
           if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
           tc_fence_after();
           const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(tr.stage * 2 * NCOLS + NCOLS + half * CW);
-          float* slot = amax + ((int64_t)lt * NI + half * (CW / G)) * kTileKeys + quad * 32 + lane;
+          // this tile's running maxima come in with the first chunk (one wait covers both loads)
+          const uint32_t am_addr = tmem_base + lane_addr + amax_col0 + (uint32_t)(lt * NI + half * NIH);
+          uint32_t am[NIH / AC][AC];
+#pragma unroll
+          for (int q = 0; q < NIH / AC; ++q) tmem_issue<AC>(am_addr + (uint32_t)(q * AC), am[q]);
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
             uint32_t r[CHK];
             tmem_issue<CHK>(taddr + (uint32_t)(c * CHK), r);
             tmem_wait<CHK>(r);
+            if (c == 0) {
+#pragma unroll
+              for (int q = 0; q < NIH / AC; ++q) tmem_wait<AC>(am[q]);
+            }
             if (c + 1 == NCH) {
               tc_fence_before();
               __syncwarp();
@@ -836,16 +906,19 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
               const float4 v = off2[c * (CHK / 4) + j];
               o[4 * j] = v.x; o[4 * j + 1] = v.y; o[4 * j + 2] = v.z; o[4 * j + 3] = v.w;
             }
-            // running max over (layer, head) of q.k - lse/c
+            // running max over (layer, head) of q.k - lse/c (slots past n_lookahead hold padding and are never read)
 #pragma unroll
             for (int ii = 0; ii < CHK / G; ++ii) {
               float mx = __uint_as_float(r[ii * G]) - o[ii * G];
 #pragma unroll
               for (int g = 1; g < G; ++g) mx = fmaxf(mx, __uint_as_float(r[ii * G + g]) - o[ii * G + g]);
               const int i = c * (CHK / G) + ii;
-              if (half * (CW / G) + i < a.n_lookahead) slot[i * kTileKeys] = fmaxf(slot[i * kTileKeys], mx);
+              am[i / AC][i % AC] = __float_as_uint(fmaxf(__uint_as_float(am[i / AC][i % AC]), mx));
             }
           }
+#pragma unroll
+          for (int q = 0; q < NIH / AC; ++q) tmem_store<AC>(am_addr + (uint32_t)(q * AC), am[q]);
+          tmem_store_wait();
         }
         if (!ok) break;
         __syncwarp();
@@ -854,17 +927,26 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       }
     }
     // ---------------- importance: mean over lookahead of exp2(c * running max) ----------------
+    tc_fence_before();
     if (ok) ok = es.sync(lane, ab);
+    tc_fence_after();
     if (ok && misc[0] == 0) {
+      // the four warps of a TMEM lane quadrant share its tiles; a thread reads all lookahead slots of its key
+      constexpr int FC = NI < 16 ? NI : 16;
       const float inv_m = 1.f / (float)a.n_lookahead;
-      for (int idx = et; idx < my_tiles * kTileKeys; idx += EW * 32) {
-        const int lt = idx / kTileKeys, kk = idx % kTileKeys;
-        const int64_t key = (int64_t)(cta + lt * n_cta) * kTileKeys + kk;
-        if (key < a.n_tokens) {
-          float s = 0.f;
-          for (int i = 0; i < a.n_lookahead; ++i) s += fast_exp2(amax[((int64_t)lt * NI + i) * kTileKeys + kk] * a.c);
-          a.importance[key] = s * inv_m;
+      for (int lt = (warp - 4) >> 2; lt < my_tiles; lt += EW / 4) {
+        const int64_t key = (int64_t)(cta + lt * n_cta) * kTileKeys + quad * 32 + lane;
+        float sacc = 0.f;
+#pragma unroll
+        for (int q = 0; q < NI / FC; ++q) {
+          uint32_t v[FC];
+          tmem_issue<FC>(tmem_base + lane_addr + amax_col0 + (uint32_t)(lt * NI + q * FC), v);
+          tmem_wait<FC>(v);
+#pragma unroll
+          for (int j = 0; j < FC; ++j)
+            if (q * FC + j < a.n_lookahead) sacc += fast_exp2(__uint_as_float(v[j]) * a.c);
         }
+        if (key < a.n_tokens) a.importance[key] = sacc * inv_m;
       }
     }
   }
@@ -904,7 +986,7 @@ EncodeTiledFn encode_fn() {
 
 struct FusedPlan {
   bool ok = false;
-  int ncols = 0, k_stages = 0, tiles_per_cta_max = 0, n_cta = 0, n_tiles = 0;
+  int ncols = 0, k_stages = 0, t_stages = 0, tiles_per_cta_max = 0, n_cta = 0, n_tiles = 0;
   SmemLayout lay{};
 };
 
@@ -922,6 +1004,11 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
   pl.n_tiles = (int)ceil_div(p.n_tokens, kTileKeys);
   pl.n_cta = std::min(std::min(sm_count, kFusedMaxCtas), pl.n_tiles);
   pl.tiles_per_cta_max = (int)ceil_div(pl.n_tiles, pl.n_cta);
+  // tensor memory: as many accumulator stages (4 at most, 2 at least) as leave room for the running maxima
+  const int amax_cols = pl.tiles_per_cta_max * (pl.ncols / g);
+  for (int ts = kTmemStages; ts >= 2 && pl.t_stages == 0; --ts)
+    if (ts * 2 * pl.ncols + amax_cols <= kTmemColsAll) pl.t_stages = ts;
+  if (pl.t_stages == 0) return pl;
   for (int ks = 10; ks >= 2; --ks) {
     const SmemLayout lay = smem_layout(p.head_dim, pl.ncols, g, ks, pl.tiles_per_cta_max);
     if ((int)lay.total <= kSmemBudget) {
@@ -1070,6 +1157,7 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   args.tiles_per_cta_max = pl.tiles_per_cta_max;
   args.lag = fused_lag(p, n_slabs);
   args.k_stages = pl.k_stages;
+  args.t_stages = pl.t_stages;
   args.c = p.c_log2;
   args.inv_c = 1.0f / p.c_log2;
   args.limbs = reinterpret_cast<unsigned long long*>(base + w.limbs_off);

@@ -195,6 +195,38 @@ SPF_API int32_t spf_compact_spans(const int32_t* kept_chunks, int64_t k, int32_t
  */
 SPF_API int64_t spf_keep_count(int64_t n_chunks, double keep_ratio);
 
+/*
+ * Host helpers for the keep rate of Section 3.1.  The keep rate is defined on the TARGET model's tokenisation:
+ * rho = compressed target length / original target length, per sample.  The paper picks compressed lengths that
+ * are whole KV-cache blocks of the serving system (8k, 16k, 24k, 32k tokens with 4k-token blocks).
+ *
+ * spf_keep_rate:        min(1, budget_tokens / target_tokens); 0 if target_tokens < 1 or budget_tokens < 1.
+ * spf_snap_budget:      the largest multiple of block_tokens that is <= desired_tokens, at least one block;
+ *                       0 if block_tokens < 1 or desired_tokens < 1.
+ * Pure host arithmetic.
+ */
+SPF_API double spf_keep_rate(int64_t target_tokens, int64_t budget_tokens);
+SPF_API int64_t spf_snap_budget(int64_t desired_tokens, int64_t block_tokens);
+
+/*
+ * ConcatWithDelim of Algorithm 1 (Section 3.2, Appendix A.3): builds the compressed prompt text from the character
+ * spans that spf_compact_spans produced.  Host routine, host pointers throughout.
+ *
+ *   text, text_bytes     the prompt as UTF-8 (need not be NUL-terminated)
+ *   char_spans           int32 [n_spans][2], half-open [start, end) in CHARACTERS (Unicode code points, as a
+ *                        tokenizer's offset mapping counts them), ascending and non-overlapping
+ *   delim, delim_bytes   UTF-8 delimiter (e.g. "[...]" or "// omitted"); written between consecutive spans only,
+ *                        never before the first or after the last; may be empty
+ *   out, out_capacity    receives the compressed text (not NUL-terminated); may be NULL with capacity 0 to query
+ *
+ * Returns the number of bytes of the compressed text.  Nothing is written unless out_capacity is at least that.
+ * A negative return is a status code: SPF_ERR_INVALID_ARG for null / negative arguments, spans that are not
+ * ascending, overlap or reach beyond the text's last character.  Bytes of the form 10xxxxxx are counted as
+ * continuations of the preceding character; the text is not otherwise validated.
+ */
+SPF_API int64_t spf_concat_with_delim(const char* text, int64_t text_bytes, const int32_t* char_spans, int64_t n_spans,
+                                      const char* delim, int64_t delim_bytes, char* out, int64_t out_capacity);
+
 /* Text of a status code (static storage). */
 SPF_API const char* spf_status_string(int32_t status);
 /* Text of the calling thread's most recent failure ("" if none).  Thread-local storage. */

@@ -6,9 +6,12 @@ from .spf_oracle import (  # noqa: F401
     chunk_means,
     compact,
     compress,
+    concat_with_delim,
     keep_count,
+    keep_rate,
     merge_adjacent,
     select_topk,
+    snap_budget,
     softmax_rows,
     token_importance,
 )

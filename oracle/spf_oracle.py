@@ -170,3 +170,25 @@ def compress(q_bits, k_bits, token_ids, char_start, char_end, *, chunk: int, kee
     ids, pos, tok_spans, char_spans = compact(kept, chunk, n, token_ids, char_start, char_end)
     return dict(importance=importance, lse=lse, chunk_scores=cs, k=k, kept=kept, ids=ids, pos=pos,
                 tok_spans=tok_spans, char_spans=char_spans)
+
+
+def keep_rate(target_tokens: int, budget_tokens: int) -> float:
+    """Section 3.1: rho = compressed target length / original target length, at most 1 (0 for empty inputs)."""
+    if target_tokens < 1 or budget_tokens < 1:
+        return 0.0
+    return min(1.0, budget_tokens / target_tokens)
+
+
+def snap_budget(desired_tokens: int, block_tokens: int) -> int:
+    """Section 3.1: compressed lengths are whole KV-cache blocks: the largest multiple of the block that is
+    at most the desired length, and at least one block (0 for empty inputs)."""
+    if desired_tokens < 1 or block_tokens < 1:
+        return 0
+    return max(1, desired_tokens // block_tokens) * block_tokens
+
+
+def concat_with_delim(text: str, char_spans: Sequence[Sequence[int]], delim: str) -> str:
+    """ConcatWithDelim of Algorithm 1 (Section 3.2, Appendix A.3): the spans' characters in order, the delimiter
+    between consecutive spans only.  Python strings index by code point, which is how a tokenizer's offset mapping
+    counts characters."""
+    return delim.join(text[int(a):int(b)] for a, b in char_spans)

@@ -58,6 +58,12 @@ def _load() -> ctypes.CDLL:
     dll.spf_compact_spans.argtypes = [vp, i64, i32, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     dll.spf_keep_count.restype = i64
     dll.spf_keep_count.argtypes = [i64, ctypes.c_double]
+    dll.spf_keep_rate.restype = ctypes.c_double
+    dll.spf_keep_rate.argtypes = [i64, i64]
+    dll.spf_snap_budget.restype = i64
+    dll.spf_snap_budget.argtypes = [i64, i64]
+    dll.spf_concat_with_delim.restype = i64
+    dll.spf_concat_with_delim.argtypes = [ctypes.c_char_p, i64, vp, i64, ctypes.c_char_p, i64, vp, i64]
     dll.spf_status_string.restype = ctypes.c_char_p
     dll.spf_status_string.argtypes = [i32]
     dll.spf_last_error.restype = ctypes.c_char_p
@@ -104,6 +110,29 @@ def spf_last_error() -> str:
 
 def spf_keep_count(n_chunks: int, keep_ratio: float) -> int:
     return int(lib.spf_keep_count(n_chunks, keep_ratio))
+
+
+def spf_keep_rate(target_tokens: int, budget_tokens: int) -> float:
+    return float(lib.spf_keep_rate(target_tokens, budget_tokens))
+
+
+def spf_snap_budget(desired_tokens: int, block_tokens: int = 4096) -> int:
+    return int(lib.spf_snap_budget(desired_tokens, block_tokens))
+
+
+def spf_concat_with_delim(text: str, char_spans, delim: str) -> str:
+    """Compressed prompt text from character spans (host routine of the library; spans as [n, 2] integers)."""
+    import numpy as np
+    raw, d = text.encode("utf-8"), delim.encode("utf-8")
+    spans = np.ascontiguousarray(np.asarray(char_spans, dtype=np.int32).reshape(-1, 2))
+    need = int(lib.spf_concat_with_delim(raw, len(raw), spans.ctypes.data, len(spans), d, len(d), None, 0))
+    if need < 0:
+        _check(need, "spf_concat_with_delim")
+    out = ctypes.create_string_buffer(max(need, 1))
+    got = int(lib.spf_concat_with_delim(raw, len(raw), spans.ctypes.data, len(spans), d, len(d), out, need))
+    if got != need:
+        _check(got if got < 0 else -1, "spf_concat_with_delim")
+    return out.raw[:need].decode("utf-8")
 
 
 @dataclasses.dataclass

@@ -97,14 +97,30 @@ SPF_API size_t spf_score_workspace_bytes(const spf_shape* shape, const spf_promp
  * on one stream.
  * `dev_status`: device int32, may be NULL.  Kernels store a negative spf_status there when a
  * device-side condition occurs (SPF_ERR_TIMEOUT from a bounded wait; SPF_ERR_RANGE when, in the fused
- * path, some logit exceeds the sampled reference of its row by more than 2^187 and the row sum
- * overflows -- the importance is then invalid and the call should be repeated on the general path);
+ * path, some logit lies more than about 50 base-2 units above the sampled reference of its (layer,
+ * kv-head) and a row sum overflows, or a row's logits all lie more than 186 units below it and the row
+ * sums to zero -- the importance is then invalid and the call should be repeated on the general path);
  * they never trap.  The caller zeroes it before the call and reads it after synchronising.
  * Errors: SPF_ERR_INVALID_ARG, SPF_ERR_UNSUPPORTED (d not 64/128, Hq % Hkv != 0, m > 32,
  * G * roundup(m,8) > 64, L > 128), SPF_ERR_WORKSPACE, SPF_ERR_CUDA.
  */
 SPF_API int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace,
                           size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * spf_score with a larger softmax denominator -- a switch for a point the paper leaves open (Section 3 describes the
+ * attention of each lookahead step "over the prompt", Appendix A.1.1 slices it to the prompt length): in the draft
+ * model, lookahead step i also attends to the i - 1 tokens generated before it and to itself, so its probabilities
+ * over the prompt sum to less than 1.  `extra_lse` is a HOST array of n_prompts DEVICE pointers (an entry may be
+ * NULL), each fp32 [L][Hq][m]: the natural log of sum exp(scale * q.k) over those non-prompt keys of row (l, h, i),
+ * as the draft model's attention kernel reports it.  Then
+ *     p[l,h,i,s] = exp(z[l,h,i,s]) / (sum_{s'} exp(z[l,h,i,s']) + exp(extra_lse[l,h,i]))
+ * and everything downstream is unchanged; prompts[p].lse receives the log of the whole denominator.  With
+ * extra_lse == NULL, or all entries NULL, this is spf_score.  Arguments, workspace and errors as for spf_score.
+ */
+SPF_API int32_t spf_score_extra(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts,
+                                const float* const* extra_lse, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                void* cuda_stream);
 
 /*
  * Chooses the kernels behind spf_score, process-wide: 0 = automatic (the fused single-kernel path when
@@ -188,6 +204,23 @@ SPF_API int32_t spf_compact_spans(const int32_t* kept_chunks, int64_t k, int32_t
                                   const int32_t* token_ids, const int32_t* char_start, const int32_t* char_end,
                                   int32_t* out_ids, int32_t* out_pos, int32_t* out_tok_spans,
                                   int32_t* out_char_spans, int64_t* out_counts, void* cuda_stream);
+
+/*
+ * Variants for two points the paper leaves open (Algorithm 1 names the operations, Appendix A.3 gives kernel 13 and
+ * the chunk sizes, nothing else).  Same arguments, layouts and errors as the calls they extend.
+ *
+ * spf_chunk_pool_edge: edge_rule 0 is spf_chunk_pool (every window is divided by pool_kernel, tokens beyond the
+ *   prompt's ends count as zeros); edge_rule 1 divides each window by the number of tokens it really covers, so
+ *   the first and last pool_kernel/2 tokens are not damped.  Other values: SPF_ERR_INVALID_ARG.
+ * spf_select_topk_forced: the first and / or the last chunk (system prompt / attention sink, and the question at
+ *   the end of the prompt) are kept whatever their scores; they count towards k, the remaining k - forced are
+ *   the best of the other chunks, ties to the lower index.  k smaller than the number of forced chunks:
+ *   SPF_ERR_INVALID_ARG.  With both flags 0 it is spf_select_topk.
+ */
+SPF_API int32_t spf_chunk_pool_edge(const float* importance, int64_t n_tokens, int32_t pool_kernel, int32_t chunk,
+                                    int32_t edge_rule, float* chunk_scores, void* cuda_stream);
+SPF_API int32_t spf_select_topk_forced(const float* chunk_scores, int64_t n_chunks, int64_t k, int32_t force_first,
+                                       int32_t force_last, int32_t* kept_chunks, void* cuda_stream);
 
 /*
  * Host helper for the keep rate of Section 3.1: the number of chunks a keep rate rho retains,

@@ -11,6 +11,7 @@ from .spf_oracle import (  # noqa: F401
     keep_rate,
     merge_adjacent,
     select_topk,
+    select_topk_forced,
     snap_budget,
     softmax_rows,
     token_importance,

@@ -59,8 +59,8 @@ def softmax_rows(z: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     return e / tot, (zmax + np.log(tot))[:, 0]
 
 
-def token_importance(q_bits: np.ndarray, k_bits: Sequence[np.ndarray], scale: Optional[float] = None
-                     ) -> Tuple[np.ndarray, np.ndarray]:
+def token_importance(q_bits: np.ndarray, k_bits: Sequence[np.ndarray], scale: Optional[float] = None,
+                     extra_lse: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
     """Max-mean aggregation of lookahead attention (Appendix A.1.1).
 
     q_bits: uint16 [L, Hq, m, d] (bf16 patterns of the post-RoPE lookahead queries)
@@ -69,6 +69,9 @@ def token_importance(q_bits: np.ndarray, k_bits: Sequence[np.ndarray], scale: Op
         p[l,h,i,:] = softmax_s(scale * Q[l,h,i] . K[l, h // G, s])
         A[i,s]     = max over all (l,h) of p[l,h,i,s]          (max over layer and head first)
         I[s]       = mean over i of A[i,s]                      (then mean over lookahead)
+    extra_lse (optional, [L, Hq, m]): the natural log of what each row's softmax denominator holds besides the
+    prompt keys (the lookahead step's own and earlier generated tokens -- a reading of a point the paper leaves
+    open); then p = exp(z) / (sum_s exp(z) + exp(extra_lse)) and the returned lse is the log of that denominator.
     """
     L, Hq, m, d = q_bits.shape
     Hkv, N, d2 = k_bits[0].shape
@@ -84,6 +87,10 @@ def token_importance(q_bits: np.ndarray, k_bits: Sequence[np.ndarray], scale: Op
             for g in range(G):
                 h = hk * G + g
                 p, lse[l, h] = softmax_rows(attention_logits(bf16_to_f64(q_bits[l, h]), k_lh, scale))
+                if extra_lse is not None:
+                    whole = np.logaddexp(lse[l, h], np.asarray(extra_lse, dtype=np.float64)[l, h])
+                    p = p * np.exp(lse[l, h] - whole)[:, None]      # the prompt's share of the larger denominator
+                    lse[l, h] = whole
                 np.maximum(A, p, out=A)
     return A.mean(axis=0), lse
 
@@ -134,6 +141,19 @@ def select_topk(chunk_scores: np.ndarray, k: int) -> np.ndarray:
 # Section 3.2 -- merge adjacent chunks, map draft-token ranges to text spans
 # (Algorithm 1: MergeAdjacentChunks, MapDraftChunksToTextSpans)
 # --------------------------------------------------------------------------------------
+def select_topk_forced(chunk_scores: np.ndarray, k: int, force_first: bool = False, force_last: bool = False) -> np.ndarray:
+    """TopKChunks with the first and / or last chunk kept whatever their scores (a reading of a point the paper
+    leaves open): the forced chunks count towards k, the other k - forced are the best of the rest, ties to the
+    lower index; ascending."""
+    n = len(chunk_scores)
+    forced = sorted({0} if force_first else set()) + ([n - 1] if force_last and not (force_first and n == 1) else [])
+    if k < len(forced):
+        raise ValueError("k is smaller than the number of forced chunks")
+    rest = [j for j in range(n) if j not in forced]
+    rest.sort(key=lambda j: (-float(chunk_scores[j]), j))        # stable: ties keep the lower index first
+    return np.array(sorted(forced + rest[:k - len(forced)]), dtype=np.int64)
+
+
 def merge_adjacent(kept: np.ndarray, c: int, n_tokens: int) -> np.ndarray:
     """Maximal runs of consecutive kept chunk indices -> token ranges [a, b), b clipped to N."""
     spans: List[Tuple[int, int]] = []

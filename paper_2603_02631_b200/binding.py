@@ -44,6 +44,8 @@ def _load() -> ctypes.CDLL:
     dll.spf_score_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32]
     dll.spf_score.restype = i32
     dll.spf_score.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp, ctypes.c_size_t, vp, vp]
+    dll.spf_score_extra.restype = i32
+    dll.spf_score_extra.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp, vp, ctypes.c_size_t, vp, vp]
     dll.spf_selftest_bounded_wait.restype = i32
     dll.spf_selftest_bounded_wait.argtypes = [vp, vp]
     dll.spf_set_score_path.restype = i32
@@ -54,6 +56,10 @@ def _load() -> ctypes.CDLL:
     dll.spf_chunk_pool.argtypes = [vp, i64, i32, i32, vp, vp]
     dll.spf_select_topk.restype = i32
     dll.spf_select_topk.argtypes = [vp, i64, i64, vp, vp]
+    dll.spf_chunk_pool_edge.restype = i32
+    dll.spf_chunk_pool_edge.argtypes = [vp, i64, i32, i32, i32, vp, vp]
+    dll.spf_select_topk_forced.restype = i32
+    dll.spf_select_topk_forced.argtypes = [vp, i64, i64, i32, i32, vp, vp]
     dll.spf_compact_spans.restype = i32
     dll.spf_compact_spans.argtypes = [vp, i64, i32, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     dll.spf_keep_count.restype = i64
@@ -195,6 +201,25 @@ def spf_score(prompts: Sequence[PromptBuffers], workspace: torch.Tensor, softmax
            "spf_score")
 
 
+def spf_score_extra(prompts: Sequence[PromptBuffers], extra_lse: Sequence[Optional[torch.Tensor]], workspace: torch.Tensor,
+                    softmax_scale: float = 0.0, dev_status: Optional[torch.Tensor] = None,
+                    stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_score with a per-row extra term in the softmax denominator: extra_lse[p] is fp32 [L, Hq, m] or None."""
+    shape, arr, _keep = _marshal(prompts, softmax_scale)
+    if len(extra_lse) != len(prompts):
+        raise ValueError("one extra_lse entry per prompt")
+    L, Hq, m, _ = prompts[0].q.shape
+    for e in extra_lse:
+        if e is not None:
+            _dev(e, torch.float32, "extra_lse")
+            if e.numel() != L * Hq * m or not e.is_contiguous():
+                raise ValueError("extra_lse must be contiguous fp32 [L, Hq, m]")
+    ptrs = (ctypes.c_void_p * len(prompts))(*[None if e is None else e.data_ptr() for e in extra_lse])
+    _check(lib.spf_score_extra(ctypes.byref(shape), arr, len(prompts), ptrs, workspace.data_ptr(),
+                               workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
+           "spf_score_extra")
+
+
 def spf_selftest_bounded_wait(dev_status: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
     """Enqueues the bounded-wait self-test; dev_status (int32, zeroed) reads SPF_ERR_TIMEOUT (-5) afterwards."""
     _dev(dev_status, torch.int32, "dev_status")
@@ -225,6 +250,29 @@ def spf_chunk_pool(importance: torch.Tensor, pool_kernel: int, chunk: int, chunk
         raise ValueError("chunk_scores is too small")
     _check(lib.spf_chunk_pool(importance.data_ptr(), n, pool_kernel, chunk, chunk_scores.data_ptr(),
                               _stream_ptr(stream)), "spf_chunk_pool")
+
+
+def spf_chunk_pool_edge(importance: torch.Tensor, pool_kernel: int, chunk: int, edge_rule: int, chunk_scores: torch.Tensor,
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_chunk_pool with the pooling edge rule as an argument (0: divide by the kernel, 1: by the tokens covered)."""
+    _dev(importance, torch.float32, "importance")
+    _dev(chunk_scores, torch.float32, "chunk_scores")
+    n = importance.numel()
+    if chunk >= 1 and chunk_scores.numel() < (n + chunk - 1) // chunk:
+        raise ValueError("chunk_scores is too small")
+    _check(lib.spf_chunk_pool_edge(importance.data_ptr(), n, pool_kernel, chunk, edge_rule, chunk_scores.data_ptr(),
+                                   _stream_ptr(stream)), "spf_chunk_pool_edge")
+
+
+def spf_select_topk_forced(chunk_scores: torch.Tensor, n_chunks: int, k: int, force_first: bool, force_last: bool,
+                           kept_chunks: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_select_topk that always keeps the first and / or the last chunk (they count towards k)."""
+    _dev(chunk_scores, torch.float32, "chunk_scores")
+    _dev(kept_chunks, torch.int32, "kept_chunks")
+    if chunk_scores.numel() < n_chunks or kept_chunks.numel() < k:
+        raise ValueError("chunk_scores or kept_chunks is too small")
+    _check(lib.spf_select_topk_forced(chunk_scores.data_ptr(), n_chunks, k, int(bool(force_first)), int(bool(force_last)),
+                                      kept_chunks.data_ptr(), _stream_ptr(stream)), "spf_select_topk_forced")
 
 
 def spf_select_topk(chunk_scores: torch.Tensor, n_chunks: int, k: int, kept_chunks: torch.Tensor,
@@ -292,9 +340,11 @@ class Selector:
 
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n_lookahead: int,
                  max_tokens: int, chunk: int = 32, pool_kernel: int = 13, softmax_scale: float = 0.0,
-                 device: str = "cuda"):
+                 device: str = "cuda", pool_edge_rule: int = 0, force_first: bool = False, force_last: bool = False):
         self.geom = (n_layers, n_q_heads, n_kv_heads, head_dim, n_lookahead)
         self.chunk, self.pool_kernel, self.softmax_scale = chunk, pool_kernel, softmax_scale
+        # switches for points the paper leaves open (defaults: the readings the library takes)
+        self.pool_edge_rule, self.force_first, self.force_last = pool_edge_rule, force_first, force_last
         self.max_tokens = max_tokens
         self.device = torch.device(device)
         max_chunks = (max_tokens + chunk - 1) // chunk
@@ -328,8 +378,16 @@ class Selector:
         k = spf_keep_count(n_chunks, keep)
         bufs = PromptBuffers(q, k_layers, self.importance[:n], self.lse)
         spf_score([bufs], self._workspace(bufs), self.softmax_scale, self.dev_status, stream)
-        spf_chunk_pool(self.importance[:n], self.pool_kernel, self.chunk, self.chunk_scores[:n_chunks], stream)
-        spf_select_topk(self.chunk_scores, n_chunks, k, self.kept, stream)
+        if self.pool_edge_rule:
+            spf_chunk_pool_edge(self.importance[:n], self.pool_kernel, self.chunk, self.pool_edge_rule,
+                                self.chunk_scores[:n_chunks], stream)
+        else:
+            spf_chunk_pool(self.importance[:n], self.pool_kernel, self.chunk, self.chunk_scores[:n_chunks], stream)
+        if self.force_first or self.force_last:
+            k = max(k, len({0} if self.force_first else set()) + (1 if self.force_last and (n_chunks > 1 or not self.force_first) else 0))
+            spf_select_topk_forced(self.chunk_scores, n_chunks, k, self.force_first, self.force_last, self.kept, stream)
+        else:
+            spf_select_topk(self.chunk_scores, n_chunks, k, self.kept, stream)
         spf_compact_spans(self.kept, k, self.chunk, n, token_ids, char_start, char_end, self.out_ids, self.out_pos,
                           self.tok_spans, self.char_spans, self.counts, stream)
         L, Hq, _, _, m = self.geom

@@ -64,6 +64,7 @@ int32_t make_problem(const spf_shape* shape, const spf_prompt& pr, int32_t index
   p.q = static_cast<const __nv_bfloat16*>(pr.q);
   p.importance = pr.importance;
   p.lse_out = pr.lse;
+  p.extra_lse = nullptr;
   *out = p;
   return SPF_OK;
 }
@@ -111,8 +112,8 @@ extern "C" size_t spf_score_workspace_bytes(const spf_shape* shape, const spf_pr
   return need;
 }
 
-extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace,
-                             size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+static int32_t score_impl(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, const float* const* extra_lse,
+                          void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
   clear_error();
   if (shape == nullptr || prompts == nullptr || n_prompts < 1)
     return fail(SPF_ERR_INVALID_ARG, "spf_score: null argument or n_prompts < 1");
@@ -137,6 +138,7 @@ extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, 
   for (int32_t i = 0; i < n_prompts; ++i) {
     ScoreProblem p;
     make_problem(shape, prompts[i], i, &p);
+    if (extra_lse != nullptr) p.extra_lse = extra_lse[i];
     const int path = g_score_path.load(std::memory_order_relaxed);
     const bool fused = path == 2 || (path == 0 && score_fused_supported(p, sm_count));
     const int32_t st = fused ? score_fused_launch(p, workspace, sm_count, dev_status, stream)
@@ -144,6 +146,17 @@ extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, 
     if (st != SPF_OK) return st;
   }
   return SPF_OK;
+}
+
+extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace,
+                             size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  return score_impl(shape, prompts, n_prompts, nullptr, workspace, workspace_bytes, dev_status, cuda_stream);
+}
+
+extern "C" int32_t spf_score_extra(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts,
+                                   const float* const* extra_lse, void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                   void* cuda_stream) {
+  return score_impl(shape, prompts, n_prompts, extra_lse, workspace, workspace_bytes, dev_status, cuda_stream);
 }
 
 extern "C" int32_t spf_selftest_bounded_wait(int32_t* dev_status, void* cuda_stream) {

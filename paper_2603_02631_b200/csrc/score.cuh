@@ -15,6 +15,7 @@ struct ScoreProblem {
   const __nv_bfloat16* q;
   float* importance;
   float* lse_out;  // may be null
+  const float* extra_lse;  // may be null: fp32 [L][Hq][m], natural log of what the row's denominator holds besides the prompt keys
 };
 
 constexpr int kMmaMaxSplit = 64;  // upper bound on the key splits of sweep 1 (sizes the partials buffer)

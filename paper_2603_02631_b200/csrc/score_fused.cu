@@ -80,6 +80,7 @@ struct FusedArgs {
   unsigned long long* limbs;  // [slab][NCOLS][kLimbStride] exact fixed-point sums of exp2(c*q.k - ref) over all keys
   unsigned* counters;     // [slab] CTAs whose share of the slab's row sums is in the accumulators
   float* lse_out;         // optional [L][Hq][m], natural log
+  const float* extra_lse; // optional [L][Hq][m], natural log: what each row's denominator holds besides the prompt keys
   float* importance;      // [N]
   int32_t* dev_status;    // optional
 };
@@ -637,10 +638,17 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
           const float mant = (float)__longlong_as_double((tb & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
           float lse2 = ref + ((float)expo + log2f(mant));
           if (!(total > 0.0) || expo == 1024) lse2 = INFINITY;  // an empty or overflowed row sum
+          const int64_t out_idx = ((int64_t)slab * G + row % G) * a.n_lookahead + row / G;
+          if (a.extra_lse != nullptr) {
+            // the denominator also holds exp(extra): log2-add, in the order that cannot overflow
+            const float e = __ldg(a.extra_lse + out_idx) * kLog2e;
+            const float hi = fmaxf(lse2, e), lo = fminf(lse2, e);
+            lse2 = hi + log2f(1.f + exp2f(lo - hi));
+          }
           if (!(lse2 > -INFINITY && lse2 < INFINITY) && a.dev_status != nullptr)
             atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
           value[r] = lse2 * a.inv_c;                            // lse in q.k units
-          if (cta == 0 && a.lse_out != nullptr) a.lse_out[((int64_t)slab * G + row % G) * a.n_lookahead + row / G] = lse2 * kLn2;
+          if (cta == 0 && a.lse_out != nullptr) a.lse_out[out_idx] = lse2 * kLn2;
         }
       }
       if (use > 0) {
@@ -1163,6 +1171,7 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   args.limbs = reinterpret_cast<unsigned long long*>(base + w.limbs_off);
   args.counters = reinterpret_cast<unsigned*>(base + w.counters_off);
   args.lse_out = p.lse_out;
+  args.extra_lse = p.extra_lse;
   args.importance = p.importance;
   args.dev_status = dev_status;
 

@@ -220,7 +220,7 @@ __global__ void __launch_bounds__(kThreads) score_lse_kernel(LayerPtrs kp, const
 
 // Merges the per-CTA partials of sweep 1: lse2[slab][row] = M + log2(Z); optional natural-log copy for the caller.
 __global__ void merge_lse_kernel(const float2* __restrict__ partial, float* __restrict__ lse2, float* __restrict__ lse_out,
-                                 int n_split, int rows_pad, int n_kv_heads, int group, int n_lookahead, int m_pad) {
+                                 const float* __restrict__ extra_lse, int n_split, int rows_pad, int n_kv_heads, int group, int n_lookahead, int m_pad) {
   const int slab = blockIdx.x;
   const int row = threadIdx.x;
   if (row >= rows_pad) return;
@@ -231,13 +231,19 @@ __global__ void merge_lse_kernel(const float2* __restrict__ partial, float* __re
     const float2 p = partial[((int64_t)slab * n_split + s) * rows_pad + row];
     z += p.y * exp2f(p.x - m);
   }
-  const float v = m + log2f(z);
-  lse2[(int64_t)slab * rows_pad + row] = v;
+  float v = m + log2f(z);
   const int g = row / m_pad, i = row % m_pad;
-  if (lse_out != nullptr && g < group && i < n_lookahead) {
-    const int layer = slab / n_kv_heads, hk = slab % n_kv_heads;
-    lse_out[(((int64_t)layer * n_kv_heads + hk) * group + g) * n_lookahead + i] = v * kLn2;
+  const int layer = slab / n_kv_heads, hk = slab % n_kv_heads;
+  const int64_t out_idx = (((int64_t)layer * n_kv_heads + hk) * group + g) * n_lookahead + i;
+  const bool real = g < group && i < n_lookahead;
+  if (extra_lse != nullptr && real) {
+    // the denominator also holds exp(extra): log2-add, in the order that cannot overflow
+    const float e = extra_lse[out_idx] * kLog2e;
+    const float hi = fmaxf(v, e), lo = fminf(v, e);
+    v = hi + log2f(1.f + exp2f(lo - hi));
   }
+  lse2[(int64_t)slab * rows_pad + row] = v;
+  if (lse_out != nullptr && real) lse_out[out_idx] = v * kLn2;
 }
 
 // Sweep 2.  One warp owns 32 keys for all slabs.  NI = m_pad / 8 lookahead indices live in a thread.
@@ -332,7 +338,7 @@ void launch_both(const ScoreProblem& p, const uint4* qf, float2* partial, float*
   const int rows_pad = p.rows_pad;
   const int n_slabs = p.n_layers * p.n_kv_heads;
   auto merge = [&]() {
-    merge_lse_kernel<<<n_slabs, 64, 0, stream>>>(partial, lse2, p.lse_out, n_split, rows_pad, p.n_kv_heads, p.group,
+    merge_lse_kernel<<<n_slabs, 64, 0, stream>>>(partial, lse2, p.lse_out, p.extra_lse, n_split, rows_pad, p.n_kv_heads, p.group,
                                                  p.n_lookahead, p.m_pad);
   };
   switch (rows_pad / 16) {

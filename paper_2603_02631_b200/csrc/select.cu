@@ -12,7 +12,7 @@ namespace {
 constexpr int kPoolWarps = 8;
 
 __global__ void __launch_bounds__(kPoolWarps * 32) chunk_pool_kernel(const float* __restrict__ importance, int64_t n_tokens,
-                                                                      int half, float inv_w, int chunk,
+                                                                      int half, float inv_w, int chunk, bool in_range_divisor,
                                                                       float* __restrict__ chunk_scores, int64_t n_chunks) {
   const int lane = threadIdx.x & 31;
   const int64_t j = (int64_t)blockIdx.x * kPoolWarps + (threadIdx.x >> 5);
@@ -24,7 +24,8 @@ __global__ void __launch_bounds__(kPoolWarps * 32) chunk_pool_kernel(const float
     const int64_t a = max(s - half, (int64_t)0), b = min(s + half, n_tokens - 1);
     float win = 0.f;
     for (int64_t t = a; t <= b; ++t) win += __ldg(importance + t);
-    sum += win * inv_w;
+    // the window's divisor: always w (zeros beyond the ends), or the number of tokens it really covers
+    sum += in_range_divisor ? win / (float)(b - a + 1) : win * inv_w;
   }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
@@ -42,6 +43,12 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   x += 0.0f;  // -0 -> +0 so that the two zeros tie
   const uint32_t b = __float_as_uint(x);
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Key of chunk j: forced chunks (bit 0 of `force`: the first chunk, bit 1: the last) sort above every score.
+__device__ __forceinline__ uint32_t chunk_key(const float* __restrict__ scores, int j, int n, int force) {
+  if (((force & 1) && j == 0) || ((force & 2) && j == n - 1)) return 0xFFFFFFFFu;
+  return order_key(scores[j]);
 }
 
 // Exclusive prefix count of `flag` over the CTA (thread order); *total gets the CTA-wide count.
@@ -62,7 +69,7 @@ __device__ __forceinline__ int block_exclusive_count(bool flag, int* warp_counts
   return before + within;
 }
 
-__global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* __restrict__ scores, int n, int k,
+__global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* __restrict__ scores, int n, int k, int force,
                                                                     int32_t* __restrict__ kept) {
   __shared__ int hist[256];
   __shared__ int warp_counts[kTopkThreads / 32];
@@ -77,7 +84,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
     for (int b = threadIdx.x; b < 256; b += kTopkThreads) hist[b] = 0;
     __syncthreads();
     for (int j = threadIdx.x; j < n; j += kTopkThreads) {
-      const uint32_t key = order_key(scores[j]);
+      const uint32_t key = chunk_key(scores, j, n, force);
       if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
     }
     __syncthreads();
@@ -126,7 +133,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   int out_base = 0, eq_base = 0;
   for (int j0 = 0; j0 < n; j0 += kTopkThreads) {
     const int j = j0 + threadIdx.x;
-    const uint32_t key = j < n ? order_key(scores[j]) : 0u;
+    const uint32_t key = j < n ? chunk_key(scores, j, n, force) : 0u;
     const bool gt = j < n && key > prefix;
     const bool eq = j < n && key == prefix;
     int eq_total, sel_total;
@@ -218,8 +225,8 @@ __global__ void __launch_bounds__(kCompactThreads) compact_spans_kernel(
 
 using namespace spf;
 
-extern "C" int32_t spf_chunk_pool(const float* importance, int64_t n_tokens, int32_t pool_kernel, int32_t chunk,
-                                  float* chunk_scores, void* cuda_stream) {
+static int32_t chunk_pool_launch(const float* importance, int64_t n_tokens, int32_t pool_kernel, int32_t chunk,
+                                 bool in_range_divisor, float* chunk_scores, void* cuda_stream) {
   clear_error();
   if (importance == nullptr || chunk_scores == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool: null pointer");
   if (n_tokens < 1) return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool: n_tokens must be >= 1 (got %lld)", (long long)n_tokens);
@@ -230,13 +237,27 @@ extern "C" int32_t spf_chunk_pool(const float* importance, int64_t n_tokens, int
   const int64_t blocks = ceil_div(n_chunks, kPoolWarps);
   if (blocks > 0x7fffffff) return fail(SPF_ERR_UNSUPPORTED, "spf_chunk_pool: too many chunks");
   chunk_pool_kernel<<<(unsigned)blocks, kPoolWarps * 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      importance, n_tokens, pool_kernel / 2, 1.0f / (float)pool_kernel, chunk, chunk_scores, n_chunks);
+      importance, n_tokens, pool_kernel / 2, 1.0f / (float)pool_kernel, chunk, in_range_divisor, chunk_scores, n_chunks);
   SPF_CUDA_CHECK(cudaGetLastError());
   return SPF_OK;
 }
 
-extern "C" int32_t spf_select_topk(const float* chunk_scores, int64_t n_chunks, int64_t k, int32_t* kept_chunks,
-                                   void* cuda_stream) {
+extern "C" int32_t spf_chunk_pool(const float* importance, int64_t n_tokens, int32_t pool_kernel, int32_t chunk,
+                                  float* chunk_scores, void* cuda_stream) {
+  return chunk_pool_launch(importance, n_tokens, pool_kernel, chunk, false, chunk_scores, cuda_stream);
+}
+
+extern "C" int32_t spf_chunk_pool_edge(const float* importance, int64_t n_tokens, int32_t pool_kernel, int32_t chunk,
+                                       int32_t edge_rule, float* chunk_scores, void* cuda_stream) {
+  if (edge_rule != 0 && edge_rule != 1) {
+    clear_error();
+    return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool_edge: edge_rule must be 0 or 1 (got %d)", edge_rule);
+  }
+  return chunk_pool_launch(importance, n_tokens, pool_kernel, chunk, edge_rule == 1, chunk_scores, cuda_stream);
+}
+
+static int32_t select_topk_launch(const float* chunk_scores, int64_t n_chunks, int64_t k, int force, int32_t* kept_chunks,
+                                  void* cuda_stream) {
   clear_error();
   if (chunk_scores == nullptr || kept_chunks == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_select_topk: null pointer");
   if (n_chunks < 1 || n_chunks > 0x7fffffff)
@@ -244,10 +265,23 @@ extern "C" int32_t spf_select_topk(const float* chunk_scores, int64_t n_chunks, 
   if (k < 1 || k > n_chunks)
     return fail(SPF_ERR_INVALID_ARG, "spf_select_topk: k must be in [1, n_chunks] (got k=%lld, n_chunks=%lld)", (long long)k,
                 (long long)n_chunks);
-  select_topk_kernel<<<1, kTopkThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(chunk_scores, (int)n_chunks, (int)k,
+  const int n_forced = (force & 1) + ((force & 2) && (n_chunks > 1 || !(force & 1)) ? 1 : 0);
+  if (k < n_forced)
+    return fail(SPF_ERR_INVALID_ARG, "spf_select_topk_forced: k = %lld is smaller than the %d forced chunks", (long long)k, n_forced);
+  select_topk_kernel<<<1, kTopkThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(chunk_scores, (int)n_chunks, (int)k, force,
                                                                                     kept_chunks);
   SPF_CUDA_CHECK(cudaGetLastError());
   return SPF_OK;
+}
+
+extern "C" int32_t spf_select_topk(const float* chunk_scores, int64_t n_chunks, int64_t k, int32_t* kept_chunks,
+                                   void* cuda_stream) {
+  return select_topk_launch(chunk_scores, n_chunks, k, 0, kept_chunks, cuda_stream);
+}
+
+extern "C" int32_t spf_select_topk_forced(const float* chunk_scores, int64_t n_chunks, int64_t k, int32_t force_first,
+                                          int32_t force_last, int32_t* kept_chunks, void* cuda_stream) {
+  return select_topk_launch(chunk_scores, n_chunks, k, (force_first ? 1 : 0) | (force_last ? 2 : 0), kept_chunks, cuda_stream);
 }
 
 extern "C" int32_t spf_compact_spans(const int32_t* kept_chunks, int64_t k, int32_t chunk, int64_t n_tokens,

@@ -180,3 +180,33 @@ def test_score_extra_matches_oracle(path):
             assert torch.equal(imp2, imp3)
     finally:
         spf.spf_set_score_path(previous)
+
+
+@pytest.mark.gpu
+def test_selector_with_all_switches_on():
+    """The chained path with the in-range pooling divisor and both ends forced, against the oracle's steps."""
+    import paper_2603_02631_b200 as spf
+    from workloads import bf16_bits, make_prompt, small_config
+    cfg = small_config("switches", n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=64, n_lookahead=8, lengths=(6000,),
+                       chunk=32, rank=4, n_needles=4, n_strong=2, needle_len=(8, 64), seed=21)
+    prompt = make_prompt(cfg, 0, "cuda")
+    n = prompt.n_tokens
+    imp, _ = oracle.token_importance(bf16_bits(prompt.q), [bf16_bits(x) for x in prompt.k])
+    scores = oracle.chunk_means(oracle.avg_pool(imp, 13, count_include_pad=False), 32)
+    k = oracle.keep_count(len(scores), 0.1)
+    kept = oracle.select_topk_forced(scores, k, True, True)
+    ids, pos, tok, ch = oracle.compact(kept, 32, n, *(t.cpu().numpy().astype(np.int64) for t in
+                                                     (prompt.token_ids, prompt.char_start, prompt.char_end)))
+    sel = spf.Selector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, n, chunk=32,
+                       pool_edge_rule=1, force_first=True, force_last=True)
+    got = sel.run(prompt.q, prompt.k, prompt.token_ids, prompt.char_start, prompt.char_end, 0.1).host()
+    np.testing.assert_allclose(got["chunk_scores"], scores, rtol=1e-3)
+    assert 0 in got["kept"] and len(scores) - 1 in got["kept"]
+    # the kept set may differ from the oracle's only inside the tie band of the k-th score among the unforced chunks
+    differ = np.setxor1d(got["kept"], kept)
+    if len(differ):
+        rest = np.sort(np.delete(scores, [0, len(scores) - 1]))[::-1]
+        tau = rest[k - 3]
+        assert (np.abs(scores[differ] - tau) <= 1e-3 * abs(tau)).all()
+    else:
+        assert np.array_equal(got["ids"], ids) and np.array_equal(got["char_spans"], ch)

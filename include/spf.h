@@ -123,6 +123,38 @@ SPF_API int32_t spf_score_extra(const spf_shape* shape, const spf_prompt* prompt
                                 void* cuda_stream);
 
 /*
+ * spf_score on a PAGED key cache (Section 3.1: the paper's serving system keeps KV caches in 4k-token blocks; a draft
+ * model served the same way has its prompt keys scattered over a block pool).  Same computation as spf_score.
+ *
+ *   k_pools        HOST array of L device pointers; layer l's pool is bf16 [n_pool_blocks][Hkv][block_tokens][d],
+ *                  contiguous, 16-byte aligned, post-RoPE
+ *   block_tokens   tokens per block, a positive multiple of 128
+ *   block_table    DEVICE int32 [ceil(N / block_tokens)]: logical block b of the prompt is pool block block_table[b].
+ *                  Entries must lie in [0, n_pool_blocks); the kernels cannot report a bad entry, but its keys then
+ *                  read as zeros (or, for the one sampled reference key, from a clamped block) instead of faulting.
+ *                  Rows of the last block beyond n_tokens are never used.
+ *   q, importance, lse   as in spf_prompt
+ *
+ * Only the fused kernel reads paged caches: shapes outside it (see spf_set_score_path) return SPF_ERR_UNSUPPORTED.
+ * Workspace: spf_score_paged_workspace_bytes(...), rules as for spf_score.  dev_status as for spf_score
+ * (on SPF_ERR_RANGE gather the keys into a contiguous cache and use spf_score's general path).
+ */
+typedef struct {
+  int64_t n_tokens;
+  const void* const* k_pools;
+  int64_t n_pool_blocks;
+  int32_t block_tokens;
+  const int32_t* block_table;
+  const void* q;
+  float* importance;
+  float* lse;
+} spf_paged_prompt;
+
+SPF_API size_t spf_score_paged_workspace_bytes(const spf_shape* shape, const spf_paged_prompt* prompts, int32_t n_prompts);
+SPF_API int32_t spf_score_paged(const spf_shape* shape, const spf_paged_prompt* prompts, int32_t n_prompts, void* workspace,
+                                size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
  * Chooses the kernels behind spf_score, process-wide: 0 = automatic (the fused single-kernel path when
  * the shape allows it, else the general two-sweep path), 1 = always the general path, 2 = always the
  * fused path (spf_score then returns SPF_ERR_UNSUPPORTED for shapes outside it: G not in {1,2,4,8},

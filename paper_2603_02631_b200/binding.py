@@ -34,6 +34,12 @@ class _Prompt(ctypes.Structure):
                 ("importance", ctypes.c_void_p), ("lse", ctypes.c_void_p)]
 
 
+class _PagedPrompt(ctypes.Structure):
+    _fields_ = [("n_tokens", ctypes.c_int64), ("k_pools", ctypes.POINTER(ctypes.c_void_p)),
+                ("n_pool_blocks", ctypes.c_int64), ("block_tokens", ctypes.c_int32), ("block_table", ctypes.c_void_p),
+                ("q", ctypes.c_void_p), ("importance", ctypes.c_void_p), ("lse", ctypes.c_void_p)]
+
+
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2603_02631_b200.build` "
@@ -46,6 +52,10 @@ def _load() -> ctypes.CDLL:
     dll.spf_score.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp, ctypes.c_size_t, vp, vp]
     dll.spf_score_extra.restype = i32
     dll.spf_score_extra.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), i32, vp, vp, ctypes.c_size_t, vp, vp]
+    dll.spf_score_paged_workspace_bytes.restype = ctypes.c_size_t
+    dll.spf_score_paged_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_PagedPrompt), i32]
+    dll.spf_score_paged.restype = i32
+    dll.spf_score_paged.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_PagedPrompt), i32, vp, ctypes.c_size_t, vp, vp]
     dll.spf_selftest_bounded_wait.restype = i32
     dll.spf_selftest_bounded_wait.argtypes = [vp, vp]
     dll.spf_set_score_path.restype = i32
@@ -218,6 +228,59 @@ def spf_score_extra(prompts: Sequence[PromptBuffers], extra_lse: Sequence[Option
     _check(lib.spf_score_extra(ctypes.byref(shape), arr, len(prompts), ptrs, workspace.data_ptr(),
                                workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
            "spf_score_extra")
+
+
+@dataclasses.dataclass
+class PagedPromptBuffers:
+    """Device buffers of one prompt whose keys sit in a block pool (see spf_paged_prompt in include/spf.h)."""
+    q: torch.Tensor                      # bf16 [L, Hq, m, d]
+    k_pools: Sequence[torch.Tensor]      # L tensors bf16 [n_pool_blocks, Hkv, block_tokens, d], contiguous
+    block_table: torch.Tensor            # int32 [ceil(N / block_tokens)]
+    n_tokens: int
+    importance: torch.Tensor             # fp32 [N] (out)
+    lse: Optional[torch.Tensor] = None   # fp32 [L, Hq, m] (out)
+
+
+def _marshal_paged(prompts: Sequence[PagedPromptBuffers], softmax_scale: float):
+    L, Hq, m, d = prompts[0].q.shape
+    Hkv = prompts[0].k_pools[0].shape[1]
+    shape = _Shape(L, Hq, Hkv, d, m, float(softmax_scale))
+    arr = (_PagedPrompt * len(prompts))()
+    keep = []
+    for i, p in enumerate(prompts):
+        _dev(p.q, torch.bfloat16, "q")
+        _dev(p.block_table, torch.int32, "block_table")
+        _dev(p.importance, torch.float32, "importance")
+        if len(p.k_pools) != L or not p.q.is_contiguous() or not p.block_table.is_contiguous():
+            raise ValueError("one contiguous pool per layer, contiguous q and block_table")
+        nb, hk, bt, dd = p.k_pools[0].shape
+        for pool in p.k_pools:
+            _dev(pool, torch.bfloat16, "k_pools[l]")
+            if tuple(pool.shape) != (nb, hk, bt, dd) or not pool.is_contiguous() or hk != Hkv or dd != d:
+                raise ValueError("every pool must be contiguous bf16 [n_pool_blocks, Hkv, block_tokens, d]")
+        if p.block_table.numel() < (p.n_tokens + bt - 1) // bt or p.importance.numel() != p.n_tokens:
+            raise ValueError("block_table or importance has the wrong size")
+        ptrs = (ctypes.c_void_p * L)(*[pool.data_ptr() for pool in p.k_pools])
+        keep.append(ptrs)
+        arr[i] = _PagedPrompt(p.n_tokens, ctypes.cast(ptrs, ctypes.POINTER(ctypes.c_void_p)), nb, bt, p.block_table.data_ptr(),
+                              p.q.data_ptr(), p.importance.data_ptr(), _ptr(p.lse))
+    return shape, arr, keep
+
+
+def spf_score_paged_workspace_bytes(prompts: Sequence[PagedPromptBuffers], softmax_scale: float = 0.0) -> int:
+    shape, arr, _keep = _marshal_paged(prompts, softmax_scale)
+    n = int(lib.spf_score_paged_workspace_bytes(ctypes.byref(shape), arr, len(prompts)))
+    if n == 0:
+        raise SpfError(-1, "spf_score_paged_workspace_bytes", spf_last_error())
+    return n
+
+
+def spf_score_paged(prompts: Sequence[PagedPromptBuffers], workspace: torch.Tensor, softmax_scale: float = 0.0,
+                    dev_status: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> None:
+    shape, arr, _keep = _marshal_paged(prompts, softmax_scale)
+    _check(lib.spf_score_paged(ctypes.byref(shape), arr, len(prompts), workspace.data_ptr(),
+                               workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
+           "spf_score_paged")
 
 
 def spf_selftest_bounded_wait(dev_status: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:

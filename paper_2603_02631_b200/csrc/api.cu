@@ -65,6 +65,9 @@ int32_t make_problem(const spf_shape* shape, const spf_prompt& pr, int32_t index
   p.importance = pr.importance;
   p.lse_out = pr.lse;
   p.extra_lse = nullptr;
+  p.block_table = nullptr;
+  p.block_tokens = 0;
+  p.n_pool_blocks = 0;
   *out = p;
   return SPF_OK;
 }
@@ -157,6 +160,79 @@ extern "C" int32_t spf_score_extra(const spf_shape* shape, const spf_prompt* pro
                                    const float* const* extra_lse, void* workspace, size_t workspace_bytes, int32_t* dev_status,
                                    void* cuda_stream) {
   return score_impl(shape, prompts, n_prompts, extra_lse, workspace, workspace_bytes, dev_status, cuda_stream);
+}
+
+// Paged key cache: the prompt is described as a contiguous one over its pool (same checks), then re-pointed at the blocks.
+static int32_t make_paged_problem(const spf_shape* shape, const spf_paged_prompt& pp, int32_t index, ScoreProblem* out) {
+  if (pp.block_tokens < 128 || pp.block_tokens % 128 != 0)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score_paged: prompt %d: block_tokens must be a positive multiple of 128 (got %d)", index,
+                pp.block_tokens);
+  if (pp.n_pool_blocks < 1 || pp.block_table == nullptr)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score_paged: prompt %d: empty pool or null block table", index);
+  if (shape == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_score_paged: null shape");
+  spf_prompt flat{};
+  flat.n_tokens = pp.n_tokens;
+  flat.k_layers = pp.k_pools;
+  flat.k_stride_tok = shape->head_dim;
+  flat.k_stride_head = (int64_t)pp.block_tokens * shape->head_dim;
+  flat.q = pp.q;
+  flat.importance = pp.importance;
+  flat.lse = pp.lse;
+  const int32_t st = make_problem(shape, flat, index, out);
+  if (st != SPF_OK) return st;
+  if (ceil_div(pp.n_tokens, pp.block_tokens) > 0x7fffffffLL) return fail(SPF_ERR_UNSUPPORTED, "spf_score_paged: too many blocks");
+  out->block_table = pp.block_table;
+  out->block_tokens = pp.block_tokens;
+  out->n_pool_blocks = pp.n_pool_blocks;
+  return SPF_OK;
+}
+
+extern "C" size_t spf_score_paged_workspace_bytes(const spf_shape* shape, const spf_paged_prompt* prompts, int32_t n_prompts) {
+  clear_error();
+  if (shape == nullptr || prompts == nullptr || n_prompts < 1) {
+    fail(SPF_ERR_INVALID_ARG, "spf_score_paged_workspace_bytes: null argument or n_prompts < 1");
+    return 0;
+  }
+  size_t need = 0;
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    if (make_paged_problem(shape, prompts[i], i, &p) != SPF_OK) return 0;
+    need = std::max(need, score_fused_workspace_bytes(p));
+  }
+  return need;
+}
+
+extern "C" int32_t spf_score_paged(const spf_shape* shape, const spf_paged_prompt* prompts, int32_t n_prompts, void* workspace,
+                                   size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  clear_error();
+  if (shape == nullptr || prompts == nullptr || n_prompts < 1)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score_paged: null argument or n_prompts < 1");
+  int sm_count = 0;
+  {
+    const int32_t st = device_sm_count(&sm_count);
+    if (st != SPF_OK) return st;
+  }
+  size_t need = 0;
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    const int32_t st = make_paged_problem(shape, prompts[i], i, &p);
+    if (st != SPF_OK) return st;
+    if (!score_fused_supported(p, sm_count))
+      return fail(SPF_ERR_UNSUPPORTED, "spf_score_paged: prompt %d: shape outside the fused kernel (the only one that reads paged caches)", i);
+    need = std::max(need, score_fused_workspace_bytes(p));
+  }
+  if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
+    return fail(SPF_ERR_WORKSPACE, "spf_score_paged: workspace is null or not 256-byte aligned");
+  if (workspace_bytes < need)
+    return fail(SPF_ERR_WORKSPACE, "spf_score_paged: workspace has %zu bytes, %zu needed", workspace_bytes, need);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    make_paged_problem(shape, prompts[i], i, &p);
+    const int32_t st = score_fused_launch(p, workspace, sm_count, dev_status, stream);
+    if (st != SPF_OK) return st;
+  }
+  return SPF_OK;
 }
 
 extern "C" int32_t spf_selftest_bounded_wait(int32_t* dev_status, void* cuda_stream) {

@@ -16,6 +16,11 @@ struct ScoreProblem {
   float* importance;
   float* lse_out;  // may be null
   const float* extra_lse;  // may be null: fp32 [L][Hq][m], natural log of what the row's denominator holds besides the prompt keys
+  // paged key cache (block_tokens > 0): k.p[l] is layer l's block pool, bf16 [n_pool_blocks][Hkv][block_tokens][d];
+  // logical block b of the prompt sits in pool block block_table[b] (device memory)
+  const int32_t* block_table;
+  int32_t block_tokens;
+  int64_t n_pool_blocks;
 };
 
 constexpr int kMmaMaxSplit = 64;  // upper bound on the key splits of sweep 1 (sizes the partials buffer)

@@ -83,6 +83,10 @@ struct FusedArgs {
   const float* extra_lse; // optional [L][Hq][m], natural log: what each row's denominator holds besides the prompt keys
   float* importance;      // [N]
   int32_t* dev_status;    // optional
+  // paged key cache: block_tokens > 0, k_layers[l] is the pool of layer l, stride_block elements between pool blocks
+  const int32_t* block_table;
+  int block_tokens;
+  int64_t stride_block, n_pool_blocks;
 };
 
 // ---------------------------------------------------------------------------------------------- PTX
@@ -196,6 +200,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                                 uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar), "l"(policy)
       : "memory");
 }
 // L2 eviction priorities for the key tiles: the first visit's tile is read again `lag` slabs later (keep it), the
@@ -368,7 +379,7 @@ __device__ __forceinline__ void tmem_wait<32>(uint32_t (&r)[32]) {
 __host__ __device__ constexpr int q_sub_tile_bytes(int ncols) { return ncols * 128; }   // ncols query rows x 64 bf16
 
 struct SmemLayout {
-  uint32_t k_off, q_off, xbuf_off, ref_off, rowoff_off, bar_off, misc_off, total;
+  uint32_t k_off, q_off, xbuf_off, ref_off, rowoff_off, tileblk_off, bar_off, misc_off, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, int k_stages, int tiles_per_cta_max) {
@@ -379,6 +390,7 @@ __host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, i
   s.xbuf_off = o;     o += (uint32_t)ncols * (kTileKeys / 4) * 4;
   s.ref_off = o;      o += kRefSlots * 4;
   s.rowoff_off = o;   o += 4 * 64 * 4;
+  s.tileblk_off = o;  o += ((uint32_t)tiles_per_cta_max * 4 + 15u) & ~15u;
   s.bar_off = o;      o += 64 * 8;
   s.misc_off = o;     o += 64;
   s.total = o;
@@ -463,6 +475,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   unsigned char* q_tiles = smem + lay.q_off;
   float* xbuf = reinterpret_cast<float*>(smem + lay.xbuf_off);         // [NCOLS][32]: partial row sums of one slab, each over four keys
   float* ref_slots = reinterpret_cast<float*>(smem + lay.ref_off);   // [kRefSlots]: slab references, kept until the log-sum-exp warp has used them
+  int* tile_block = reinterpret_cast<int*>(smem + lay.tileblk_off);   // paged key cache: pool block of each of the CTA's tiles
   float* rowoff = reinterpret_cast<float*>(smem + lay.rowoff_off);   // [4 slots][64]: what the epilogue subtracts per row
   volatile int* misc = reinterpret_cast<volatile int*>(smem + lay.misc_off);  // [0] abort, [1] tmem base, [3] references written
   const Bars bars{smem_u32(smem + lay.bar_off), a.k_stages};
@@ -503,6 +516,10 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     mbar_init(bars.x_free(), EWV);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // paged key cache: a tile never straddles a block (blocks are multiples of 128 tokens), one lookup per tile for the whole kernel
+  if (a.block_tokens > 0)
+    for (int lt = threadIdx.x; lt < my_tiles; lt += kThreads)
+      tile_block[lt] = a.block_table[(int64_t)(cta + lt * n_cta) * kTileKeys / a.block_tokens];
   // zero the query stages: rows the TMA box does not cover must read as zero
   for (uint32_t i = threadIdx.x * 16; i < (uint32_t)kQStages * 2 * kQSlotBytes; i += kThreads * 16)
     *reinterpret_cast<uint4*>(q_tiles + i) = make_uint4(0, 0, 0, 0);
@@ -546,9 +563,13 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
           for (int v = 0; v < 2; ++v) {
             if (!valid[v]) continue;
             const int layer = slab_of[v] / a.n_kv_heads, hk = slab_of[v] % a.n_kv_heads;
-            for (int h = 0; h < KSUB; ++h)
-              tma_load_3d(smem_u32(k_tiles + kr.stage * kStageBytes + v * kSlotBytes + h * kSubTileBytes), &maps.k[layer],
-                          h * 64, key0, hk, bars.k_full(kr.stage), policy[v]);
+            for (int h = 0; h < KSUB; ++h) {
+              const uint32_t dst = smem_u32(k_tiles + kr.stage * kStageBytes + v * kSlotBytes + h * kSubTileBytes);
+              if (a.block_tokens > 0)
+                tma_load_4d_hint(dst, &maps.k[layer], h * 64, key0 % a.block_tokens, hk, tile_block[lt], bars.k_full(kr.stage), policy[v]);
+              else
+                tma_load_3d(dst, &maps.k[layer], h * 64, key0, hk, bars.k_full(kr.stage), policy[v]);
+            }
           }
           kr.advance();
         }
@@ -669,12 +690,20 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     // and reports this CTA (keeps the fence off the epilogue warps) =====
     bool ok = true;
     const int64_t sample_key = a.n_tokens / 2;                  // the same key for every CTA: one reference per slab
+    // where that key sits: its row inside its pool block when the cache is paged (a bad table entry is clamped: this is a
+    // plain load, not a bounds-checked TMA copy)
+    int64_t sample_block = 0, sample_row = sample_key;
+    if (a.block_tokens > 0) {
+      sample_block = min(max((int64_t)__ldg(a.block_table + sample_key / a.block_tokens), (int64_t)0), a.n_pool_blocks - 1);
+      sample_row = sample_key % a.block_tokens;
+    }
     for (int slab = 0; ok && slab < n_slabs + 2; ++slab) {
       if (slab < n_slabs) {
         const int x = slab & 1;
         const int use = slab >> 1;
         const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
-        const uint4* krow = reinterpret_cast<const uint4*>(a.k_layers[layer] + hk * a.stride_head + sample_key * a.stride_tok);
+        const uint4* krow = reinterpret_cast<const uint4*>(a.k_layers[layer] + sample_block * a.stride_block + hk * a.stride_head +
+                                                           sample_row * a.stride_tok);
         const uint4* qrow[2];
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
@@ -1139,7 +1168,20 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(SPF_ERR_CUDA, "spf_score: encoding the query tensor map failed (CUresult %d)", (int)r);
   }
-  for (int l = 0; l < p.n_layers; ++l) {
+  for (int l = 0; l < p.n_layers && p.block_tokens > 0; ++l) {
+    // paged: (d, row in block, kv-head, pool block); a table entry outside the pool reads as zeros instead of faulting
+    const cuuint64_t bt = (cuuint64_t)p.block_tokens;
+    const cuuint64_t dims[4] = {(cuuint64_t)d, bt, (cuuint64_t)p.n_kv_heads, (cuuint64_t)p.n_pool_blocks};
+    const cuuint64_t strides[3] = {(cuuint64_t)d * 2, bt * d * 2, (cuuint64_t)p.n_kv_heads * bt * d * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)kTileKeys, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = encode(&maps.k[l], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(p.k.p[l]), dims, strides,
+                              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+      return fail(SPF_ERR_CUDA, "spf_score_paged: encoding the key tensor map of layer %d failed (CUresult %d)", l, (int)r);
+  }
+  for (int l = 0; l < p.n_layers && p.block_tokens == 0; ++l) {
     const cuuint64_t head_stride = p.n_kv_heads > 1 ? (cuuint64_t)p.stride_head : (cuuint64_t)p.stride_tok * p.n_tokens;
     const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)p.n_tokens, (cuuint64_t)p.n_kv_heads};
     const cuuint64_t strides[2] = {(cuuint64_t)p.stride_tok * 2, head_stride * 2};
@@ -1174,6 +1216,10 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   args.extra_lse = p.extra_lse;
   args.importance = p.importance;
   args.dev_status = dev_status;
+  args.block_table = p.block_table;
+  args.block_tokens = p.block_tokens;
+  args.stride_block = (int64_t)p.n_kv_heads * p.block_tokens * p.head_dim;
+  args.n_pool_blocks = p.n_pool_blocks;
 
   SPF_CUDA_CHECK(cudaMemsetAsync(base, 0, w.total, stream));
   if (d == 64) return launch_fused_n<64>(pl.ncols, g, maps, args, pl, stream);

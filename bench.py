@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM read + write bytes of one scoring launch, from the ncu capture summarised in profiles/.  Each entry names
 # the SHA-256 of the kernel source it was taken from: once the source changes, the figure is reported as null.
 NCU_TRAFFIC = {
-    ("long128k", "fused"): {"bytes": 4 * (599572736 + 7007488), "source": "paper_2603_02631_b200/csrc/score_fused.cu",
-                            "sha256": "7c0b447ef601990b9d377a3e582d65278a2c9f08e65132994864f008bc8a5d37",
+    ("long128k", "fused"): {"bytes": 4 * (595414016 + 6846464), "source": "paper_2603_02631_b200/csrc/score_fused.cu",
+                            "sha256": "076c1bcc878ca9646bf59484c91eb3d3debc4dae6489605a35fed6af81fcf992",
                             "note": "captured on long128k_l4 (4 of 16 layers), scaled x4"},
 }
 

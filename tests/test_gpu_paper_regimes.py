@@ -68,3 +68,31 @@ def test_keep_rates_from_three_to_fifty_percent():
                        chunk=32, keep=(0.03, 0.06, 0.10, 0.25, 0.45, 0.50), rank=8, n_needles=16, n_strong=4,
                        needle_len=(16, 128), recency=True, seed=13)
     _check(cfg, cfg.keep)
+
+
+def test_two_accumulator_stages_when_the_running_maxima_need_the_room():
+    """64 query rows per kv-head and 9 key tiles per CTA: the running maxima take 144 tensor-memory columns, which
+    leaves room for two accumulator stages only (the fused kernel picks that layout by itself)."""
+    cfg = small_config("deep", n_layers=1, n_q_heads=4, n_kv_heads=1, head_dim=64, n_lookahead=16, lengths=(160001,),
+                       chunk=32, keep=(0.10,), rank=8, n_needles=16, n_strong=4, needle_len=(16, 128), seed=14)
+    _check(cfg, cfg.keep, paths=(2,))
+
+
+def test_prompt_beyond_the_fused_kernels_capacity_takes_the_general_path():
+    """17 key tiles per CTA at 64 query rows do not fit next to two accumulator stages: pinned to the fused kernel the
+    call is refused, left on automatic it is scored by the general path."""
+    import paper_2603_02631_b200 as spf
+    cfg = small_config("huge", n_layers=1, n_q_heads=4, n_kv_heads=1, head_dim=64, n_lookahead=16, lengths=(310000,),
+                       chunk=32, keep=(0.06,), rank=8, n_needles=16, n_strong=4, needle_len=(16, 128), seed=15)
+    prompt = make_prompt(cfg, 0, "cuda")
+    imp = torch.empty(prompt.n_tokens, dtype=torch.float32, device="cuda")
+    bufs = spf.PromptBuffers(prompt.q, prompt.k, imp, None)
+    ws = torch.empty(spf.spf_score_workspace_bytes([bufs]), dtype=torch.uint8, device="cuda")
+    previous = spf.spf_set_score_path(2)
+    try:
+        with pytest.raises(spf.SpfError) as err:
+            spf.spf_score([bufs], ws)
+        assert err.value.status == -2
+    finally:
+        spf.spf_set_score_path(previous)
+    _check(cfg, cfg.keep, paths=(0,))

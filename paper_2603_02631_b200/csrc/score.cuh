@@ -32,7 +32,7 @@ int32_t score_mma_launch(const ScoreProblem& p, void* workspace, int sm_count, c
 // Fused single-kernel path (tcgen05 + TMA, key cache read once from HBM).  Covers G in {1,2,4,8},
 // G*m <= 64, up to kFusedMaxLayers layers and prompt lengths whose per-CTA state fits shared memory.
 constexpr int kFusedMaxLayers = 64;
-constexpr int kFusedMaxCtas = 256;  // upper bound on the persistent grid (sizes the partials buffer)
+constexpr int kFusedMaxCtas = 256;  // upper bound on the persistent grid
 bool score_fused_supported(const ScoreProblem& p, int sm_count);
 size_t score_fused_workspace_bytes(const ScoreProblem& p);
 int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count, int32_t* dev_status, cudaStream_t stream);

@@ -54,7 +54,6 @@ namespace {
 
 constexpr int kTileKeys = 128;
 constexpr int kThreads = 640;          // warp 0 TMA, 1 MMA issue, 2 log-sum-exp, 3 references + publisher, 4..19 epilogue
-constexpr int kIssuers = 1;            // MMA-issuing warps: local tile lt belongs to issuer lt % kIssuers
 constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accumulators (covers every finite fp32)
 constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
 constexpr int kQStages = 2;
@@ -266,9 +265,8 @@ __host__ __device__ constexpr uint32_t instr_desc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileKeys >> 4) << 24);
 }
 
-// TMEM -> registers, split in two so that a load can be in flight while the previous tile is processed:
-// tmem_issue starts the (asynchronous) load of N consecutive columns of the warp's 32 lanes, tmem_wait
-// completes it.  The registers are listed as in/out operands of the wait so that no use can move above it.
+// TMEM -> registers, in two parts: tmem_issue starts the (asynchronous) load of N consecutive columns of the warp's
+// 32 lanes, tmem_wait completes every load the thread has started.  The registers are listed as in/out operands of the wait so that no use can move above it.
 template <int N>
 __device__ __forceinline__ void tmem_issue(uint32_t taddr, uint32_t (&r)[N]);
 template <int N>
@@ -415,7 +413,7 @@ struct Bars {
   __device__ uint32_t x_ready() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 10 + kPubSlots); }
   __device__ uint32_t x_free() const { return base + 8u * (2 * k_stages + 2 * kQStages + 2 * kTmemStages + 11 + kPubSlots); }
 };
-// 2 * 10 + 2 * 2 + 2 * 4 + 10 + 16 + 2 = 60 barriers at most; the block has room for 64.
+// 2 * 10 + 2 * 2 + 2 * 4 + 10 + 16 + 2 = 60 barriers at most (10 key stages, kTmemStages = 4); the block has room for 64.
 
 struct Ring {
   int stage = 0;
@@ -491,7 +489,6 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   if (threadIdx.x == 0) {
     misc[0] = 0;
     misc[1] = 0;
-    misc[2] = 0;
     misc[3] = 0;
     for (int s = 0; s < a.k_stages; ++s) {
       mbar_init(bars.k_full(s), 1);
@@ -499,7 +496,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     }
     for (int s = 0; s < kQStages; ++s) {
       mbar_init(bars.q_full(s), 1);
-      mbar_init(bars.q_empty(s), kIssuers);
+      mbar_init(bars.q_empty(s), 1);
     }
     for (int s = 0; s < a.t_stages; ++s) {
       mbar_init(bars.t_full(s), 1);
@@ -510,7 +507,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       mbar_init(bars.o_free(x), EWV);
     }
     mbar_init(bars.epi_sync(), EW);
-    mbar_init(bars.mma_done(), kIssuers);
+    mbar_init(bars.mma_done(), 1);
     for (int b = 0; b < kPubSlots; ++b) mbar_init(bars.pub_ready(b), EWV);
     mbar_init(bars.x_ready(), EWV);
     mbar_init(bars.x_free(), EWV);

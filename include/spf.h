@@ -135,9 +135,8 @@ SPF_API int32_t spf_score_extra(const spf_shape* shape, const spf_prompt* prompt
  *                  Rows of the last block beyond n_tokens are never used.
  *   q, importance, lse   as in spf_prompt
  *
- * Only the fused kernel reads paged caches: shapes outside it (see spf_set_score_path) return SPF_ERR_UNSUPPORTED.
- * Workspace: spf_score_paged_workspace_bytes(...), rules as for spf_score.  dev_status as for spf_score
- * (on SPF_ERR_RANGE gather the keys into a contiguous cache and use spf_score's general path).
+ * Both kernel paths read paged caches (spf_set_score_path applies); shapes, errors and dev_status as for spf_score.
+ * Workspace: spf_score_paged_workspace_bytes(...), rules as for spf_score.
  */
 typedef struct {
   int64_t n_tokens;

@@ -197,7 +197,7 @@ extern "C" size_t spf_score_paged_workspace_bytes(const spf_shape* shape, const 
   for (int32_t i = 0; i < n_prompts; ++i) {
     ScoreProblem p;
     if (make_paged_problem(shape, prompts[i], i, &p) != SPF_OK) return 0;
-    need = std::max(need, score_fused_workspace_bytes(p));
+    need = std::max(need, std::max(score_mma_workspace_bytes(p), score_fused_workspace_bytes(p)));
   }
   return need;
 }
@@ -217,9 +217,7 @@ extern "C" int32_t spf_score_paged(const spf_shape* shape, const spf_paged_promp
     ScoreProblem p;
     const int32_t st = make_paged_problem(shape, prompts[i], i, &p);
     if (st != SPF_OK) return st;
-    if (!score_fused_supported(p, sm_count))
-      return fail(SPF_ERR_UNSUPPORTED, "spf_score_paged: prompt %d: shape outside the fused kernel (the only one that reads paged caches)", i);
-    need = std::max(need, score_fused_workspace_bytes(p));
+    need = std::max(need, std::max(score_mma_workspace_bytes(p), score_fused_workspace_bytes(p)));
   }
   if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
     return fail(SPF_ERR_WORKSPACE, "spf_score_paged: workspace is null or not 256-byte aligned");
@@ -229,7 +227,10 @@ extern "C" int32_t spf_score_paged(const spf_shape* shape, const spf_paged_promp
   for (int32_t i = 0; i < n_prompts; ++i) {
     ScoreProblem p;
     make_paged_problem(shape, prompts[i], i, &p);
-    const int32_t st = score_fused_launch(p, workspace, sm_count, dev_status, stream);
+    const int path = g_score_path.load(std::memory_order_relaxed);
+    const bool fused = path == 2 || (path == 0 && score_fused_supported(p, sm_count));
+    const int32_t st = fused ? score_fused_launch(p, workspace, sm_count, dev_status, stream)
+                             : score_mma_launch(p, workspace, sm_count, stream);
     if (st != SPF_OK) return st;
   }
   return SPF_OK;

@@ -56,17 +56,38 @@ struct KeyTile {
   uint4 r[4][D / 32];
 };
 
+// Paged key cache (block_tokens > 0): the pointers of LayerPtrs are block pools, bf16 [blocks][Hkv][block_tokens][d];
+// logical block b of the prompt is pool block table[b].  A 32-key tile never straddles a block (blocks are multiples
+// of 128 tokens), so one table entry places a whole tile.
+struct PagedView {
+  const int32_t* table;
+  int block_tokens;
+  int64_t stride_block, n_pool_blocks;
+};
+
+// Element offset, from the (layer, kv-head) base pointer, of the row of key0 (the first key of a tile).
+__device__ __forceinline__ int64_t tile_offset(int64_t key0, int64_t stride_tok, const PagedView& pv) {
+  if (pv.block_tokens == 0) return key0 * stride_tok;
+  int64_t block = __ldg(pv.table + key0 / pv.block_tokens);
+  block = block < 0 ? 0 : (block >= pv.n_pool_blocks ? pv.n_pool_blocks - 1 : block);   // a bad entry must not fault
+  return block * pv.stride_block + (key0 % pv.block_tokens) * stride_tok;
+}
+
 template <int D>
-__device__ __forceinline__ void load_key_tile(KeyTile<D>& t, const __nv_bfloat16* slab, int64_t key0, int64_t n_tokens,
-                                              int64_t stride_tok, int lane) {
+__device__ __forceinline__ void load_key_tile(KeyTile<D>& t, const __nv_bfloat16* slab, int64_t tile_off, int64_t key0,
+                                              int64_t n_tokens, int64_t stride_tok, int lane) {
 #pragma unroll
   for (int nt = 0; nt < 4; ++nt) {
     int64_t key = key0 + nt * 8 + (lane >> 2);
-    key = key < n_tokens ? key : n_tokens - 1;  // ragged tail: read a valid row, mask later
-    const __nv_bfloat16* row = slab + key * stride_tok + (lane & 3) * 8;
+    key = key < n_tokens ? key : n_tokens - 1;  // ragged tail: read a valid row (of the same tile), mask later
+    const __nv_bfloat16* row = slab + tile_off + (key - key0) * stride_tok + (lane & 3) * 8;
 #pragma unroll
     for (int j = 0; j < D / 32; ++j) t.r[nt][j] = load_key16(row + j * 32);
   }
+}
+
+inline PagedView paged_view(const ScoreProblem& p) {
+  return PagedView{p.block_table, p.block_tokens, (int64_t)p.n_kv_heads * p.block_tokens * p.head_dim, p.n_pool_blocks};
 }
 
 // acc[mt][nt] = logits of rows 16*mt.. against keys 8*nt.. (fp32, unscaled).
@@ -131,7 +152,7 @@ template <int D, int MT>
 __global__ void __launch_bounds__(kThreads) score_lse_kernel(LayerPtrs kp, const uint4* __restrict__ qf,
                                                               float2* __restrict__ partial, int64_t n_tokens,
                                                               int64_t stride_head, int64_t stride_tok, int n_kv_heads,
-                                                              float c) {
+                                                              float c, PagedView pv) {
   const int slab = blockIdx.y;
   const int layer = slab / n_kv_heads, hk = slab % n_kv_heads;
   const __nv_bfloat16* kslab = kp.p[layer] + hk * stride_head;
@@ -148,11 +169,11 @@ __global__ void __launch_bounds__(kThreads) score_lse_kernel(LayerPtrs kp, const
 
   int64_t tile = (int64_t)blockIdx.x * kWarpsPerCta + warp;
   KeyTile<D> cur;
-  if (tile < n_tiles) load_key_tile<D>(cur, kslab, tile * kTileKeys, n_tokens, stride_tok, lane);
+  if (tile < n_tiles) load_key_tile<D>(cur, kslab, tile_offset(tile * kTileKeys, stride_tok, pv), tile * kTileKeys, n_tokens, stride_tok, lane);
   while (tile < n_tiles) {
     const int64_t next = tile + stride;
     KeyTile<D> nxt;
-    if (next < n_tiles) load_key_tile<D>(nxt, kslab, next * kTileKeys, n_tokens, stride_tok, lane);
+    if (next < n_tiles) load_key_tile<D>(nxt, kslab, tile_offset(next * kTileKeys, stride_tok, pv), next * kTileKeys, n_tokens, stride_tok, lane);
 
     float acc[MT][4][4];
     tile_logits<D, MT>(acc, cur, qslab, lane);
@@ -252,7 +273,7 @@ __global__ void __launch_bounds__(kThreads) score_max_kernel(LayerPtrs kp, const
                                                               const float* __restrict__ lse2, float* __restrict__ importance,
                                                               int64_t n_tokens, int64_t stride_head, int64_t stride_tok,
                                                               int n_layers, int n_kv_heads, int group, int n_lookahead,
-                                                              float c) {
+                                                              float c, PagedView pv) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t tile = (int64_t)blockIdx.x * kWarpsPerCta + warp;
   const int64_t n_tiles = (n_tokens + kTileKeys - 1) / kTileKeys;
@@ -267,12 +288,13 @@ __global__ void __launch_bounds__(kThreads) score_max_kernel(LayerPtrs kp, const
     for (int x = 0; x < 8; ++x) amax[s][x] = -INFINITY;
 
   KeyTile<D> cur;
-  load_key_tile<D>(cur, kp.p[0], key0, n_tokens, stride_tok, lane);
+  const int64_t tile_off = tile_offset(key0, stride_tok, pv);   // the same for every layer and kv-head
+  load_key_tile<D>(cur, kp.p[0], tile_off, key0, n_tokens, stride_tok, lane);
   for (int slab = 0; slab < n_slabs; ++slab) {
     KeyTile<D> nxt;
     if (slab + 1 < n_slabs) {
       const int l2 = (slab + 1) / n_kv_heads, h2 = (slab + 1) % n_kv_heads;
-      load_key_tile<D>(nxt, kp.p[l2] + h2 * stride_head, key0, n_tokens, stride_tok, lane);
+      load_key_tile<D>(nxt, kp.p[l2] + h2 * stride_head, tile_off, key0, n_tokens, stride_tok, lane);
     }
     float acc[MT][4][4];
     tile_logits<D, MT>(acc, cur, qf + (int64_t)slab * (MT * (D / 16) * 32), lane);
@@ -312,7 +334,7 @@ template <int D, int MT>
 void launch_lse(const ScoreProblem& p, const uint4* qf, float2* partial, int n_split, cudaStream_t stream) {
   dim3 grid(n_split, p.n_layers * p.n_kv_heads);
   score_lse_kernel<D, MT><<<grid, kThreads, 0, stream>>>(p.k, qf, partial, p.n_tokens, p.stride_head, p.stride_tok,
-                                                         p.n_kv_heads, p.c_log2);
+                                                         p.n_kv_heads, p.c_log2, paged_view(p));
 }
 
 template <int D, int MT, int NI>
@@ -320,7 +342,7 @@ void launch_max(const ScoreProblem& p, const uint4* qf, const float* lse2, cudaS
   const int64_t n_tiles = ceil_div(p.n_tokens, kTileKeys);
   score_max_kernel<D, MT, NI><<<(unsigned)ceil_div(n_tiles, kWarpsPerCta), kThreads, 0, stream>>>(
       p.k, qf, lse2, p.importance, p.n_tokens, p.stride_head, p.stride_tok, p.n_layers, p.n_kv_heads, p.group,
-      p.n_lookahead, p.c_log2);
+      p.n_lookahead, p.c_log2, paged_view(p));
 }
 
 template <int D, int MT>

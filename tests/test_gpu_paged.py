@@ -32,8 +32,17 @@ def _paged_copy(k_layers, n, block_tokens, n_spare, seed):
     (1, 4, 1, 64, 16, 50000, 128),      # one tile per block
     (1, 2, 1, 64, 8, 100, 256),         # a single, partly filled block
 ])
-def test_paged_scoring(L, Hq, Hkv, d, m, N, bt):
+@pytest.mark.parametrize("path", [2, 1])
+def test_paged_scoring(L, Hq, Hkv, d, m, N, bt, path):
     import paper_2603_02631_b200 as spf
+    outer = spf.spf_set_score_path(path)
+    try:
+        _paged_case(spf, L, Hq, Hkv, d, m, N, bt, path)
+    finally:
+        spf.spf_set_score_path(outer)
+
+
+def _paged_case(spf, L, Hq, Hkv, d, m, N, bt, path):
     cfg = small_config("paged", n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, n_lookahead=m, lengths=(N,),
                        rank=4, n_needles=2 if N >= 300 else 0, n_strong=1, needle_len=(4, 40), seed=N + bt)
     prompt = make_prompt(cfg, 0, "cuda")
@@ -52,8 +61,8 @@ def test_paged_scoring(L, Hq, Hkv, d, m, N, bt):
     rel = np.abs(got - want_imp) / np.maximum(want_imp, 1e-30)
     assert rel.max() <= 1e-3, rel.max()
     np.testing.assert_allclose(lse.cpu().numpy().reshape(L, Hq, m), want_lse, rtol=0, atol=2e-4)
-    # the same kernel on the contiguous keys: identical bits
-    previous = spf.spf_set_score_path(2)
+    # the same kernels on the contiguous keys: identical bits
+    previous = spf.spf_set_score_path(path)
     try:
         imp2 = torch.empty_like(imp)
         flat = spf.PromptBuffers(prompt.q, prompt.k, imp2, None)

@@ -437,10 +437,29 @@ class Selector:
         n = k_layers[0].shape[1]
         if n > self.max_tokens:
             raise ValueError(f"prompt has {n} tokens, selector was sized for {self.max_tokens}")
-        n_chunks = (n + self.chunk - 1) // self.chunk
-        k = spf_keep_count(n_chunks, keep)
         bufs = PromptBuffers(q, k_layers, self.importance[:n], self.lse)
         spf_score([bufs], self._workspace(bufs), self.softmax_scale, self.dev_status, stream)
+        return self._select(n, token_ids, char_start, char_end, keep, stream)
+
+    def run_paged(self, q: torch.Tensor, k_pools: Sequence[torch.Tensor], block_table: torch.Tensor, n_tokens: int,
+                  token_ids: torch.Tensor, char_start: torch.Tensor, char_end: torch.Tensor, keep: float,
+                  stream: Optional[torch.cuda.Stream] = None) -> Selection:
+        """run() for a prompt whose keys sit in a block pool (see PagedPromptBuffers)."""
+        n = n_tokens
+        if n > self.max_tokens:
+            raise ValueError(f"prompt has {n} tokens, selector was sized for {self.max_tokens}")
+        bufs = PagedPromptBuffers(q, k_pools, block_table, n, self.importance[:n], self.lse)
+        need = spf_score_paged_workspace_bytes([bufs], self.softmax_scale)
+        if self.workspace is None or self.workspace.numel() < need:
+            self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        spf_score_paged([bufs], self.workspace, self.softmax_scale, self.dev_status, stream)
+        return self._select(n, token_ids, char_start, char_end, keep, stream)
+
+    def _select(self, n: int, token_ids: torch.Tensor, char_start: torch.Tensor, char_end: torch.Tensor, keep: float,
+                stream: Optional[torch.cuda.Stream]) -> Selection:
+        """Pooling, top-k and compaction on the importance scores already in self.importance[:n]."""
+        n_chunks = (n + self.chunk - 1) // self.chunk
+        k = spf_keep_count(n_chunks, keep)
         if self.pool_edge_rule:
             spf_chunk_pool_edge(self.importance[:n], self.pool_kernel, self.chunk, self.pool_edge_rule,
                                 self.chunk_scores[:n_chunks], stream)

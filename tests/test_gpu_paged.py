@@ -84,3 +84,22 @@ def test_paged_argument_checks():
         table = torch.zeros(8, dtype=torch.int32, device="cuda")
         with pytest.raises(spf.SpfError):
             spf.spf_score_paged_workspace_bytes([spf.PagedPromptBuffers(prompt.q, pools, table, 300, imp)])
+
+
+def test_paged_selection_end_to_end():
+    """The chained path on a paged cache gives the selection the contiguous cache gives."""
+    import paper_2603_02631_b200 as spf
+    cfg = small_config("paged", n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=64, n_lookahead=8, lengths=(12345,),
+                       rank=4, n_needles=4, n_strong=2, needle_len=(8, 64), seed=31)
+    prompt = make_prompt(cfg, 0, "cuda")
+    n = prompt.n_tokens
+    pools, table = _paged_copy(prompt.k, n, 4096, n_spare=2, seed=5)
+    sel = spf.Selector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, n)
+    a = sel.run(prompt.q, prompt.k, prompt.token_ids, prompt.char_start, prompt.char_end, 0.1).host()
+    b = sel.run_paged(prompt.q, pools, table, n, prompt.token_ids, prompt.char_start, prompt.char_end, 0.1).host()
+    assert int(sel.dev_status.item()) == 0
+    for key in ("importance", "kept", "ids", "pos", "tok_spans", "char_spans"):
+        assert np.array_equal(a[key], b[key]), key
+    ref = oracle.compress(bf16_bits(prompt.q), [bf16_bits(x) for x in prompt.k], prompt.token_ids.cpu().numpy(),
+                          prompt.char_start.cpu().numpy(), prompt.char_end.cpu().numpy(), chunk=32, keep=0.1, pool_kernel=13)
+    assert np.array_equal(b["kept"], ref["kept"]) and np.array_equal(b["ids"], ref["ids"])

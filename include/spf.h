@@ -154,6 +154,27 @@ SPF_API int32_t spf_score_paged(const spf_shape* shape, const spf_paged_prompt* 
                                 size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
 
 /*
+ * One long prompt over several GPUs (Appendix A.1.1 is per prompt; this shards its keys).  Each rank holds a contiguous
+ * range of the prompt's keys for all layers and describes it as an spf_prompt of its own (n_tokens = the range's
+ * length).  A softmax row spans all ranks, so scoring takes two calls with one exchange between them:
+ *
+ *   spf_score_shard_lse     writes to prompt->lse (required) the natural-log sum-exp of every row over THIS rank's keys;
+ *                           prompt->importance is ignored.
+ *   (caller)                combines the ranks' values: lse_all = log sum_r exp(lse_r) -- e.g. a max all-reduce and a
+ *                           sum all-reduce of exp(lse_r - max), L * Hq * m floats.
+ *   spf_score_shard_apply   given lse_all (device fp32 [L][Hq][m]) writes the importance of this rank's keys, exactly
+ *                           what spf_score would give them in the whole prompt; prompt->lse is ignored.
+ *
+ * Pooling needs a halo of pool_kernel / 2 importance values from each neighbour, the top-k needs all ranks' chunk
+ * scores; both are the caller's exchanges.  These two calls use the general two-sweep kernels (one sweep each);
+ * workspace as spf_score_workspace_bytes for the shard, errors as spf_score.
+ */
+SPF_API int32_t spf_score_shard_lse(const spf_shape* shape, const spf_prompt* prompt, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream);
+SPF_API int32_t spf_score_shard_apply(const spf_shape* shape, const spf_prompt* prompt, const float* lse, void* workspace,
+                                      size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Chooses the kernels behind spf_score, process-wide: 0 = automatic (the fused single-kernel path when
  * the shape allows it, else the general two-sweep path), 1 = always the general path, 2 = always the
  * fused path (spf_score then returns SPF_ERR_UNSUPPORTED for shapes outside it: G not in {1,2,4,8},

@@ -56,6 +56,10 @@ def _load() -> ctypes.CDLL:
     dll.spf_score_paged_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_PagedPrompt), i32]
     dll.spf_score_paged.restype = i32
     dll.spf_score_paged.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_PagedPrompt), i32, vp, ctypes.c_size_t, vp, vp]
+    dll.spf_score_shard_lse.restype = i32
+    dll.spf_score_shard_lse.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), vp, ctypes.c_size_t, vp]
+    dll.spf_score_shard_apply.restype = i32
+    dll.spf_score_shard_apply.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), vp, vp, ctypes.c_size_t, vp]
     dll.spf_selftest_bounded_wait.restype = i32
     dll.spf_selftest_bounded_wait.argtypes = [vp, vp]
     dll.spf_set_score_path.restype = i32
@@ -281,6 +285,28 @@ def spf_score_paged(prompts: Sequence[PagedPromptBuffers], workspace: torch.Tens
     _check(lib.spf_score_paged(ctypes.byref(shape), arr, len(prompts), workspace.data_ptr(),
                                workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
            "spf_score_paged")
+
+
+def spf_score_shard_lse(prompt: PromptBuffers, workspace: torch.Tensor, softmax_scale: float = 0.0,
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Row log-sum-exps over this shard's keys only, written to prompt.lse (see spf_score_shard_lse in include/spf.h)."""
+    if prompt.lse is None:
+        raise ValueError("prompt.lse receives the result")
+    shape, arr, _keep = _marshal([prompt], softmax_scale)
+    _check(lib.spf_score_shard_lse(ctypes.byref(shape), arr, workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                   _stream_ptr(stream)), "spf_score_shard_lse")
+
+
+def spf_score_shard_apply(prompt: PromptBuffers, lse_all: torch.Tensor, workspace: torch.Tensor, softmax_scale: float = 0.0,
+                          stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Importance of this shard's keys given the whole prompt's row log-sum-exps (fp32 [L, Hq, m])."""
+    _dev(lse_all, torch.float32, "lse_all")
+    shape, arr, _keep = _marshal([prompt], softmax_scale)
+    L, Hq, m, _ = prompt.q.shape
+    if lse_all.numel() != L * Hq * m or not lse_all.is_contiguous():
+        raise ValueError("lse_all must be contiguous fp32 [L, Hq, m]")
+    _check(lib.spf_score_shard_apply(ctypes.byref(shape), arr, lse_all.data_ptr(), workspace.data_ptr(),
+                                     workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "spf_score_shard_apply")
 
 
 def spf_selftest_bounded_wait(dev_status: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:

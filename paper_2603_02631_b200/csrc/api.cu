@@ -236,6 +236,44 @@ extern "C" int32_t spf_score_paged(const spf_shape* shape, const spf_paged_promp
   return SPF_OK;
 }
 
+// Key-sharded scoring: the two sweeps of the general path as separate calls.
+static int32_t score_shard(const spf_shape* shape, const spf_prompt* prompt, int phase, const float* lse_in, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream, const char* who) {
+  clear_error();
+  if (shape == nullptr || prompt == nullptr) return fail(SPF_ERR_INVALID_ARG, "%s: null argument", who);
+  spf_prompt pr = *prompt;
+  float dummy = 0.f;
+  if (phase == 1) {
+    if (pr.lse == nullptr) return fail(SPF_ERR_INVALID_ARG, "%s: prompt->lse receives the result and must not be null", who);
+    pr.importance = &dummy;   // not written by this phase; only passes the null check below
+  } else if (lse_in == nullptr) {
+    return fail(SPF_ERR_INVALID_ARG, "%s: lse is null", who);
+  }
+  ScoreProblem p;
+  const int32_t st = make_problem(shape, pr, 0, &p);
+  if (st != SPF_OK) return st;
+  if (phase == 1) p.importance = nullptr;
+  if (phase == 2) p.lse_out = nullptr;
+  const size_t need = score_mma_workspace_bytes(p);
+  if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
+    return fail(SPF_ERR_WORKSPACE, "%s: workspace is null or not 256-byte aligned", who);
+  if (workspace_bytes < need) return fail(SPF_ERR_WORKSPACE, "%s: workspace has %zu bytes, %zu needed", who, workspace_bytes, need);
+  int sm_count = 0;
+  const int32_t sc = device_sm_count(&sm_count);
+  if (sc != SPF_OK) return sc;
+  return score_mma_launch_phase(p, workspace, sm_count, phase, lse_in, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int32_t spf_score_shard_lse(const spf_shape* shape, const spf_prompt* prompt, void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream) {
+  return score_shard(shape, prompt, 1, nullptr, workspace, workspace_bytes, cuda_stream, "spf_score_shard_lse");
+}
+
+extern "C" int32_t spf_score_shard_apply(const spf_shape* shape, const spf_prompt* prompt, const float* lse, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream) {
+  return score_shard(shape, prompt, 2, lse, workspace, workspace_bytes, cuda_stream, "spf_score_shard_apply");
+}
+
 extern "C" int32_t spf_selftest_bounded_wait(int32_t* dev_status, void* cuda_stream) {
   clear_error();
   if (dev_status == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_selftest_bounded_wait: dev_status is null");

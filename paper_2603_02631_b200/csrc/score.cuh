@@ -28,6 +28,10 @@ constexpr int kMmaMaxSplit = 64;  // upper bound on the key splits of sweep 1 (s
 // General two-sweep path (warp-level mma.sync tiles, key cache read twice).
 size_t score_mma_workspace_bytes(const ScoreProblem& p);
 int32_t score_mma_launch(const ScoreProblem& p, void* workspace, int sm_count, cudaStream_t stream);
+// phase 1: row log-sum-exps of the given keys only (to p.lse_out); phase 2: importance of the given keys from row
+// log-sum-exps supplied by the caller (device, natural log, [L][Hq][m]); phase 0 is score_mma_launch
+int32_t score_mma_launch_phase(const ScoreProblem& p, void* workspace, int sm_count, int phase, const float* lse_in,
+                               cudaStream_t stream);
 
 // Fused single-kernel path (tcgen05 + TMA, key cache read once from HBM).  Covers G in {1,2,4,8},
 // G*m <= 64, up to kFusedMaxLayers layers and prompt lengths whose per-CTA state fits shared memory.

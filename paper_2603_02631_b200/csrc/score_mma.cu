@@ -267,6 +267,20 @@ __global__ void merge_lse_kernel(const float2* __restrict__ partial, float* __re
   if (lse_out != nullptr && real) lse_out[out_idx] = v * kLn2;
 }
 
+// Key-sharded scoring: the row log-sum-exps of the WHOLE prompt come from the caller (natural log, [L][Hq][m]); this
+// lays them out as sweep 2 reads them (base 2, padded rows).
+__global__ void load_lse_kernel(const float* __restrict__ lse_in, float* __restrict__ lse2, int rows_pad, int n_kv_heads,
+                                int group, int n_lookahead, int m_pad) {
+  const int slab = blockIdx.x;
+  const int row = threadIdx.x;
+  if (row >= rows_pad) return;
+  const int g = row / m_pad, i = row % m_pad;
+  const int layer = slab / n_kv_heads, hk = slab % n_kv_heads;
+  float v = 0.f;
+  if (g < group && i < n_lookahead) v = lse_in[(((int64_t)layer * n_kv_heads + hk) * group + g) * n_lookahead + i] * kLog2e;
+  lse2[(int64_t)slab * rows_pad + row] = v;
+}
+
 // Sweep 2.  One warp owns 32 keys for all slabs.  NI = m_pad / 8 lookahead indices live in a thread.
 template <int D, int MT, int NI>
 __global__ void __launch_bounds__(kThreads) score_max_kernel(LayerPtrs kp, const uint4* __restrict__ qf,
@@ -355,19 +369,25 @@ void launch_max_ni(const ScoreProblem& p, const uint4* qf, const float* lse2, cu
   }
 }
 
+// phase 0: both sweeps; 1: sweep 1 and the merge only (row log-sum-exps of the keys given); 2: sweep 2 only, with the
+// row log-sum-exps `lse_in` supplied by the caller
 template <int D>
-void launch_both(const ScoreProblem& p, const uint4* qf, float2* partial, float* lse2, int n_split, cudaStream_t stream) {
+void launch_both(const ScoreProblem& p, const uint4* qf, float2* partial, float* lse2, int n_split, int phase, const float* lse_in,
+                 cudaStream_t stream) {
   const int rows_pad = p.rows_pad;
   const int n_slabs = p.n_layers * p.n_kv_heads;
   auto merge = [&]() {
     merge_lse_kernel<<<n_slabs, 64, 0, stream>>>(partial, lse2, p.lse_out, p.extra_lse, n_split, rows_pad, p.n_kv_heads, p.group,
                                                  p.n_lookahead, p.m_pad);
   };
+  if (phase == 2)
+    load_lse_kernel<<<n_slabs, 64, 0, stream>>>(lse_in, lse2, rows_pad, p.n_kv_heads, p.group, p.n_lookahead, p.m_pad);
+  const bool s1 = phase != 2, s2 = phase != 1;
   switch (rows_pad / 16) {
-    case 1: launch_lse<D, 1>(p, qf, partial, n_split, stream); merge(); launch_max_ni<D, 1>(p, qf, lse2, stream); break;
-    case 2: launch_lse<D, 2>(p, qf, partial, n_split, stream); merge(); launch_max_ni<D, 2>(p, qf, lse2, stream); break;
-    case 3: launch_lse<D, 3>(p, qf, partial, n_split, stream); merge(); launch_max_ni<D, 3>(p, qf, lse2, stream); break;
-    default: launch_lse<D, 4>(p, qf, partial, n_split, stream); merge(); launch_max_ni<D, 4>(p, qf, lse2, stream); break;
+    case 1: if (s1) { launch_lse<D, 1>(p, qf, partial, n_split, stream); merge(); } if (s2) launch_max_ni<D, 1>(p, qf, lse2, stream); break;
+    case 2: if (s1) { launch_lse<D, 2>(p, qf, partial, n_split, stream); merge(); } if (s2) launch_max_ni<D, 2>(p, qf, lse2, stream); break;
+    case 3: if (s1) { launch_lse<D, 3>(p, qf, partial, n_split, stream); merge(); } if (s2) launch_max_ni<D, 3>(p, qf, lse2, stream); break;
+    default: if (s1) { launch_lse<D, 4>(p, qf, partial, n_split, stream); merge(); } if (s2) launch_max_ni<D, 4>(p, qf, lse2, stream); break;
   }
 }
 
@@ -389,7 +409,8 @@ MmaLayout mma_layout(const ScoreProblem& p) {
 
 size_t score_mma_workspace_bytes(const ScoreProblem& p) { return mma_layout(p).total; }
 
-int32_t score_mma_launch(const ScoreProblem& p, void* workspace, int sm_count, cudaStream_t stream) {
+int32_t score_mma_launch_phase(const ScoreProblem& p, void* workspace, int sm_count, int phase, const float* lse_in,
+                               cudaStream_t stream) {
   const MmaLayout w = mma_layout(p);
   char* base = static_cast<char*>(workspace);
   uint4* qf = reinterpret_cast<uint4*>(base + w.qf_off);
@@ -405,11 +426,15 @@ int32_t score_mma_launch(const ScoreProblem& p, void* workspace, int sm_count, c
   pack_q_kernel<<<n_slabs, 128, 0, stream>>>(p.q, qf, p.n_kv_heads, p.group, p.n_lookahead, p.m_pad, p.head_dim,
                                              p.rows_pad / 16);
   if (p.head_dim == 64)
-    launch_both<64>(p, qf, partial, lse2, (int)n_split, stream);
+    launch_both<64>(p, qf, partial, lse2, (int)n_split, phase, lse_in, stream);
   else
-    launch_both<128>(p, qf, partial, lse2, (int)n_split, stream);
+    launch_both<128>(p, qf, partial, lse2, (int)n_split, phase, lse_in, stream);
   SPF_CUDA_CHECK(cudaGetLastError());
   return SPF_OK;
+}
+
+int32_t score_mma_launch(const ScoreProblem& p, void* workspace, int sm_count, cudaStream_t stream) {
+  return score_mma_launch_phase(p, workspace, sm_count, 0, nullptr, stream);
 }
 
 }  // namespace spf

@@ -11,6 +11,11 @@
  *   spf_select_topk    Appendix A.1.2 / Algorithm 1 "TopKChunks".
  *   spf_compact_spans  Section 3.2 / Algorithm 1 "MergeAdjacentChunks" + "MapDraftChunksToTextSpans".
  *
+ * Around them: spf_keep_count / spf_keep_rate / spf_snap_budget (Section 3.1, keep rate) and spf_concat_with_delim
+ * (Algorithm 1 "ConcatWithDelim") on the host; spf_score_paged (paged key cache), spf_score_shard_lse /
+ * spf_score_shard_apply (one prompt's keys over several GPUs); spf_score_extra, spf_chunk_pool_edge,
+ * spf_select_topk_forced (switches for points the paper leaves open); spf_score_static (no allocation).
+ *
  * Symbols: N prompt tokens (the paper's S), m lookahead queries (the paper's N), L layers, Hq query
  * heads (the paper's H), Hkv key heads, G = Hq / Hkv, d head dimension, c chunk size, C = ceil(N / c),
  * k chunks kept, w pooling kernel.

@@ -18,17 +18,21 @@
 // [128 keys x NCOLS rows] in tensor memory.  Keys are TMEM lanes, so an epilogue thread owns one key
 // and sees all query rows of it: the max over heads is in-thread.
 //
-// Warps.  0: TMA producer.  1: MMA issuer.  2: log-sum-exp warp (turns a slab's complete row sums into the
-// offsets of visit 2).  3: reference + publisher warp.  4..11: "sum" warps, the visit-1 half of every stage
-// (exp2-bound).  12..19: "max" warps, the visit-2 half (ALU / shared-memory bound); they also add up the per-key
-// sums of the sum warps, which reach them through a shared-memory buffer once per slab.  The two groups run
-// independently, so the exp2 work and the max work overlap on every scheduler.
+// Warps.  0: TMA producer of the first-visit tiles.  1: MMA issuer.  2: log-sum-exp warp (turns a slab's complete
+// row sums into the offsets of visit 2).  3: reference + publisher warp.  4..11: "sum" warps, the visit-1 half of
+// every stage (exp2-bound).  12..19: "max" warps, the visit-2 half (ALU / shared-memory bound); they also add up the
+// per-key sums of the sum warps, which reach them through a shared-memory buffer once per slab.  20: TMA producer of
+// the second-visit tiles.  The two epilogue groups run independently, so the exp2 work and the max work overlap on
+// every scheduler.
 //
-// Reference.  Visit 1 subtracts one reference per slab inside the exp2 argument so that exp2 cannot overflow:
-// the largest logit of the slab's rows against one fixed sample key, plus a margin of 60 (base-2 units).  Sums
-// stay finite unless some logit exceeds that sample logit by more than about 50 base-2 units; a row whose logits
-// all lie more than 186 units below it sums to zero.  Both cases are reported as SPF_ERR_RANGE (the caller can
-// then use the general path).
+// Reference.  Visit 1 subtracts one reference per slab inside the exp2 argument: the SMALLEST logit of the slab's
+// rows against one fixed sample key, plus a margin of 60 (base-2 units).  Every row's largest logit is at least
+// its own sample logit, hence at least reference - 60, and ex2.approx.ftz only flushes terms below reference - 126,
+// i.e. terms more than 2^66 times smaller than the row's largest: no row can lose anything that matters, whatever
+// the spread between the heads of a group.  What can still go wrong is overflow: a row sum reaches 2^128 when some
+// logit lies about 188 - log2(keys at that level) base-2 units (157 at the very least, about 109 nats) above the
+// slab's smallest sample logit.  That is detected (the sum is inf) and reported as SPF_ERR_RANGE; the caller can
+// then use the general path.
 //
 // Cross-CTA step.  All CTAs use the same reference for a slab, so their partial sums can simply be added.
 // To make the total independent of the order in which CTAs arrive, the fp32 partial sums are added
@@ -38,12 +42,12 @@
 // Results are bit-identical from run to run.  Because visit 1 never waits on another CTA and all CTAs are
 // co-resident, the counters always fill.
 //
-// Every wait in this file is bounded: on expiry the kernel records SPF_ERR_TIMEOUT, drains and
-// returns normally.
+// Every wait on a barrier, counter or flag in this file is bounded: on expiry the kernel records SPF_ERR_TIMEOUT,
+// drains and returns normally.  The one wait that has no limit is the hardware's own: tcgen05.alloc blocks while
+// another resident CTA on the SM holds tensor memory (this kernel asks for all of it), i.e. until that CTA exits.
 #include <cuda.h>
 
 #include <algorithm>
-#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -53,7 +57,8 @@ namespace spf {
 namespace {
 
 constexpr int kTileKeys = 128;
-constexpr int kThreads = 640;          // warp 0 TMA, 1 MMA issue, 2 log-sum-exp, 3 references + publisher, 4..19 epilogue
+constexpr int kThreads = 672;          // warp 0 TMA (first visit), 1 MMA issue, 2 log-sum-exp, 3 references + publisher, 4..19 epilogue, 20 TMA (second visit)
+constexpr int kProducer2Warp = 20;
 constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accumulators (covers every finite fp32)
 constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
 constexpr int kQStages = 2;
@@ -491,11 +496,11 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     misc[1] = 0;
     misc[3] = 0;
     for (int s = 0; s < a.k_stages; ++s) {
-      mbar_init(bars.k_full(s), 1);
+      mbar_init(bars.k_full(s), 2);            // one arrival per producer warp
       mbar_init(bars.k_empty(s), 1);
     }
     for (int s = 0; s < kQStages; ++s) {
-      mbar_init(bars.q_full(s), 1);
+      mbar_init(bars.q_full(s), 2);
       mbar_init(bars.q_empty(s), 1);
     }
     for (int s = 0; s < a.t_stages; ++s) {
@@ -533,40 +538,46 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
   const uint32_t tmem_base = (uint32_t)misc[1];
 
   // ------------------------------------------------------------------ roles
-  if (warp == 0) {
-    // ===== TMA producer: per run t the query tiles of both slabs, then per key tile of the CTA one stage holding
-    // the tile of slab t (first visit, slot 0) and the same tile of slab t - lag (second visit, slot 1) =====
+  if (warp == 0 || warp == kProducer2Warp) {
+    // ===== TMA producers.  Stage (t, j) of the key ring holds tile j of slab t (first visit, slot 0, streamed from HBM)
+    // and the same tile of slab t - lag (second visit, slot 1, normally still in L2); per run t the query tiles of both
+    // slabs go to one stage of the query ring.  One thread starts a copy only every few hundred cycles, whatever the
+    // copy's size, and a single producer thread was what bounded the whole kernel; so each visit has a producer warp of
+    // its own (warp 0: first visit, warp 20: second).  Both arrive on the stage's "full" barrier: with the byte count
+    // of their copies, or plainly where their visit has no slab (the first and last `lag` runs) =====
     if (lane == 0) {
+      const int v = warp == 0 ? 0 : 1;
       Ring kr(a.k_stages), qr(kQStages);
-      const uint64_t policy[2] = {l2_policy_keep(), l2_policy_drop()};
+      const uint64_t policy = v == 0 ? l2_policy_keep() : l2_policy_drop();
       bool ok = true;
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
-        const bool v1 = t < n_slabs, v2 = t >= a.lag;
-        const int slab_of[2] = {t, t - a.lag};
-        const bool valid[2] = {v1, v2};
+        const bool valid = v == 0 ? t < n_slabs : t >= a.lag;
+        const int slab = v == 0 ? t : t - a.lag;
         if (!(ok = mbar_wait(bars.q_empty(qr.stage), qr.phase ^ 1u, ab))) break;
-        mbar_expect_tx(bars.q_full(qr.stage), (uint32_t)(((int)v1 + (int)v2) * KSUB * rows_real * 128));
-        for (int v = 0; v < 2; ++v) {
-          if (!valid[v]) continue;
+        if (valid) {
+          mbar_expect_tx(bars.q_full(qr.stage), (uint32_t)(KSUB * rows_real * 128));
           for (int h = 0; h < KSUB; ++h)
-            tma_load_4d(smem_u32(q_tiles + (qr.stage * 2 + v) * kQSlotBytes + h * kQSub), &maps.q, h * 64, 0, 0, slab_of[v],
+            tma_load_4d(smem_u32(q_tiles + (qr.stage * 2 + v) * kQSlotBytes + h * kQSub), &maps.q, h * 64, 0, 0, slab,
                         bars.q_full(qr.stage));
+        } else {
+          mbar_arrive(bars.q_full(qr.stage));
         }
         qr.advance();
+        const int layer = valid ? slab / a.n_kv_heads : 0, hk = valid ? slab % a.n_kv_heads : 0;
         for (int lt = 0; lt < my_tiles; ++lt) {
           const int key0 = (cta + lt * n_cta) * kTileKeys;
           if (!(ok = mbar_wait(bars.k_empty(kr.stage), kr.phase ^ 1u, ab))) break;
-          mbar_expect_tx(bars.k_full(kr.stage), (uint32_t)(((int)v1 + (int)v2) * kSlotBytes));
-          for (int v = 0; v < 2; ++v) {
-            if (!valid[v]) continue;
-            const int layer = slab_of[v] / a.n_kv_heads, hk = slab_of[v] % a.n_kv_heads;
+          if (valid) {
+            mbar_expect_tx(bars.k_full(kr.stage), (uint32_t)kSlotBytes);
             for (int h = 0; h < KSUB; ++h) {
               const uint32_t dst = smem_u32(k_tiles + kr.stage * kStageBytes + v * kSlotBytes + h * kSubTileBytes);
               if (a.block_tokens > 0)
-                tma_load_4d_hint(dst, &maps.k[layer], h * 64, key0 % a.block_tokens, hk, tile_block[lt], bars.k_full(kr.stage), policy[v]);
+                tma_load_4d_hint(dst, &maps.k[layer], h * 64, key0 % a.block_tokens, hk, tile_block[lt], bars.k_full(kr.stage), policy);
               else
-                tma_load_3d(dst, &maps.k[layer], h * 64, key0, hk, bars.k_full(kr.stage), policy[v]);
+                tma_load_3d(dst, &maps.k[layer], h * 64, key0, hk, bars.k_full(kr.stage), policy);
             }
+          } else {
+            mbar_arrive(bars.k_full(kr.stage));
           }
           kr.advance();
         }
@@ -681,7 +692,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       if (lane == 0) mbar_arrive(bars.o_ready(x));
     }
   } else if (warp == 3) {
-    // ===== reference / publisher warp.  Per slab: the reference of the first visit (the largest logit of the slab's
+    // ===== reference / publisher warp.  Per slab: the reference of the first visit (the smallest logit of the slab's
     // rows against one fixed sample key, plus a margin), written as soon as the slot of slab - 2 is free; then, once
     // the shares of slab - 2 have been added to the accumulators, orders those additions before the arrival count
     // and reports this CTA (keeps the fence off the epilogue warps) =====
@@ -731,10 +742,12 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
             }
           }
         }
-        // one reference per slab: the largest sample logit of its rows (padding rows repeat a real one), base-2 units
-        float ref = fmaxf(dot[0], dot[1]);
+        // one reference per slab: the smallest sample logit of its rows (padding rows repeat a real one), in base-2
+        // units, plus the margin.  The smallest, so that no row's sum can underflow (see the header).  A softmax scale
+        // is positive, so the smallest q.k is the smallest logit
+        float ref = fminf(dot[0], dot[1]);
 #pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) ref = fmaxf(ref, __shfl_xor_sync(0xffffffffu, ref, off));
+        for (int off = 16; off >= 1; off >>= 1) ref = fminf(ref, __shfl_xor_sync(0xffffffffu, ref, off));
         ref = fmaf(ref, a.c, kRefMargin);
         if (use > 0) {
           if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
@@ -1057,16 +1070,11 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
 
 // How many slabs the second visit runs behind the first.  The cross-CTA hand-over of a slab's row sums takes
 // about 5 us; with short slabs (few tiles per CTA) two slabs of lead do not cover it, so the lag grows until the
-// slabs kept live for the second read (lag + 1 of them) would no longer sit comfortably in L2.  The
-// environment variable SPF_FUSED_LAG (1..8) overrides the choice for tuning.
+// slabs kept live for the second read (lag + 1 of them) would no longer sit comfortably in L2.
 int fused_lag(const ScoreProblem& p, int n_slabs) {
   const double slab_bytes = (double)p.n_tokens * p.head_dim * 2.0;
   int lag = (int)(80.0 * 1024 * 1024 / slab_bytes) - 1;
   lag = std::max(2, std::min(lag, 8));
-  if (const char* env = getenv("SPF_FUSED_LAG")) {
-    const int v = atoi(env);
-    if (v >= 1 && v <= 8) lag = v;
-  }
   return std::max(1, std::min(lag, n_slabs));
 }
 
@@ -1083,13 +1091,36 @@ FusedWorkspace fused_workspace(const ScoreProblem& p) {
   return w;
 }
 
+// The kernel's cross-CTA hand-over needs every CTA of the grid on an SM at the same time.  The launch therefore asks the
+// runtime for exactly that guarantee (a cooperative launch; no grid-wide barrier is used): a grid that cannot be
+// co-resident -- fewer SMs available than the device reports, e.g. under MPS with a limited SM share -- is refused
+// here instead of spinning into the bounded waits.  SMs that are merely busy with other kernels delay the launch;
+// they do not break it.
 template <int D, int NCOLS, int G>
 int32_t launch_fused(const FusedMaps& maps, const FusedArgs& args, const FusedPlan& pl, cudaStream_t stream) {
   auto kern = score_fused_kernel<D, NCOLS, G>;
   const int smem_bytes = (int)pl.lay.total + 1024;
   SPF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
-  kern<<<pl.n_cta, kThreads, smem_bytes, stream>>>(maps, args);
-  SPF_CUDA_CHECK(cudaGetLastError());
+  int per_sm = 0;
+  SPF_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, smem_bytes));
+  if (per_sm < 1) return fail(SPF_ERR_UNSUPPORTED, "spf_score: the fused kernel does not fit an SM of this device");
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)pl.n_cta);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = (size_t)smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, maps, args);
+  if (err == cudaErrorCooperativeLaunchTooLarge) {
+    (void)cudaGetLastError();
+    return fail(SPF_ERR_UNSUPPORTED, "spf_score: the %d CTAs of the fused kernel cannot all be resident on this device; use the general path",
+                pl.n_cta);
+  }
+  SPF_CUDA_CHECK(err);
   return SPF_OK;
 }
 

@@ -14,7 +14,8 @@
  * Around them: spf_keep_count / spf_keep_rate / spf_snap_budget (Section 3.1, keep rate) and spf_concat_with_delim
  * (Algorithm 1 "ConcatWithDelim") on the host; spf_score_paged (paged key cache), spf_score_shard_lse /
  * spf_score_shard_apply (one prompt's keys over several GPUs); spf_score_extra, spf_chunk_pool_edge,
- * spf_select_topk_forced (switches for points the paper leaves open); spf_score_static (no allocation).
+ * spf_select_topk_forced (switches for points the paper leaves open); spf_compress_host (the four calls for host
+ * buffers); spf_score_static (no allocation).
  *
  * Symbols: N prompt tokens (the paper's S), m lookahead queries (the paper's N), L layers, Hq query
  * heads (the paper's H), Hkv key heads, G = Hq / Hkv, d head dimension, c chunk size, C = ceil(N / c),
@@ -26,8 +27,8 @@
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work is
  *     enqueued on it; no call synchronises the stream or the device.
  *   - Return value: SPF_OK (0) or a negative spf_status.  Argument checks happen on the host before
- *     anything is launched; a failing call launches nothing.  spf_last_error() gives the text of the
- *     calling thread's last failure.
+ *     anything is launched; a call that fails them launches nothing.  spf_last_error() gives the text of
+ *     the calling thread's last failure.
  *   - Conditions only the device can see are written to `dev_status` (see spf_score).
  *   - Nothing here falls back to the CPU: unsupported shapes return SPF_ERR_UNSUPPORTED.
  */
@@ -54,7 +55,7 @@ typedef enum {
   SPF_ERR_WORKSPACE = -3,   /* workspace missing, misaligned or smaller than the size query says    */
   SPF_ERR_CUDA = -4,        /* a CUDA runtime call failed (no device, launch error)                 */
   SPF_ERR_TIMEOUT = -5,     /* device status only: a bounded wait inside a kernel ran out           */
-  SPF_ERR_RANGE = -6        /* device status only: a softmax row overflowed fp32 in the fused path  */
+  SPF_ERR_RANGE = -6        /* device status only: a softmax row sum overflowed fp32 in the fused path */
 } spf_status;
 
 /* Draft-model attention geometry shared by all prompts of a call. */
@@ -100,14 +101,26 @@ SPF_API size_t spf_score_workspace_bytes(const spf_shape* shape, const spf_promp
  * `workspace`: device, 256-byte aligned, at least spf_score_workspace_bytes(...) bytes; contents on
  * entry are irrelevant, contents on exit unspecified.  Calls that share a workspace must be ordered
  * on one stream.
- * `dev_status`: device int32, may be NULL.  Kernels store a negative spf_status there when a
- * device-side condition occurs (SPF_ERR_TIMEOUT from a bounded wait; SPF_ERR_RANGE when, in the fused
- * path, some logit lies more than about 50 base-2 units above the sampled reference of its (layer,
- * kv-head) and a row sum overflows, or a row's logits all lie more than 186 units below it and the row
- * sums to zero -- the importance is then invalid and the call should be repeated on the general path);
- * they never trap.  The caller zeroes it before the call and reads it after synchronising.
+ * `dev_status`: device int32, may be NULL (device-side conditions then go unreported).  Kernels store a
+ * negative spf_status there when a device-side condition occurs; they never trap.  The caller zeroes it
+ * before the call and reads it after synchronising.  Conditions:
+ *   SPF_ERR_TIMEOUT  a bounded wait of the fused path ran out (2 s): the kernel returned without results.
+ *                    The fused kernel needs all its CTAs resident at once and asks the runtime for that at
+ *                    launch; the wait can still run out if the GPU is shared so heavily that a hand-over
+ *                    between CTAs takes seconds.
+ *   SPF_ERR_RANGE    fused path only.  Its first sweep sums exp2(logit - r) per softmax row in fp32, with one
+ *                    reference r per (layer, kv-head): 60 base-2 units above the smallest logit that the rows of
+ *                    that kv-head have against the key at position N / 2.  No row can underflow (its largest
+ *                    term is at least 2^-60, and what is flushed is 2^66 times smaller), whatever the spread
+ *                    between the heads of a group.  A row sum overflows when some logit lies about 188 -
+ *                    log2(number of such keys) base-2 units -- 157 at the very least, about 109 nats -- above that
+ *                    smallest sample logit.  The importance is then invalid and the call should be repeated on
+ *                    the general path (spf_set_score_path(1)), which has no such limit.
  * Errors: SPF_ERR_INVALID_ARG, SPF_ERR_UNSUPPORTED (d not 64/128, Hq % Hkv != 0, m > 32,
- * G * roundup(m,8) > 64, L > 128), SPF_ERR_WORKSPACE, SPF_ERR_CUDA.
+ * G * roundup(m,8) > 64, L > 128; with the fused path forced, also shapes outside it or a grid that cannot be
+ * co-resident on the device), SPF_ERR_WORKSPACE, SPF_ERR_CUDA.  All prompts are validated before the first
+ * launch; a shape that only the forced fused path refuses is found when its prompt's turn comes, after earlier
+ * prompts of the batch have been enqueued.
  */
 SPF_API int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace,
                           size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
@@ -278,6 +291,41 @@ SPF_API int32_t spf_chunk_pool_edge(const float* importance, int64_t n_tokens, i
                                     int32_t edge_rule, float* chunk_scores, void* cuda_stream);
 SPF_API int32_t spf_select_topk_forced(const float* chunk_scores, int64_t n_chunks, int64_t k, int32_t force_first,
                                        int32_t force_last, int32_t* kept_chunks, void* cuda_stream);
+
+/*
+ * The whole path for ONE prompt whose inputs and results live in HOST memory (Algorithm 1 from AggregateMaxMean to
+ * MapDraftChunksToTextSpans): copies the inputs to the device, runs spf_score -> spf_chunk_pool -> spf_select_topk
+ * -> spf_compact_spans, copies the selection back.  This is the entry for a caller that holds the draft model's
+ * tensors on the host or on another device; a caller whose tensors are already on this GPU chains the four calls
+ * itself.  Unlike every other call it SYNCHRONISES `cuda_stream` (twice: once to learn the counts, once at the end).
+ *
+ *   k_layers_host   HOST array of L HOST pointers, layer l bf16 [Hkv][N][d] contiguous (pinned memory copies at full
+ *                   PCIe / NVLink-C2C speed, pageable memory works)
+ *   q_host          HOST bf16 [L][Hq][m][d]
+ *   token_ids_host, char_start_host, char_end_host   HOST int32 [N]
+ *   params          chunk size c, pooling kernel w (odd), keep rate rho: k = spf_keep_count(ceil(N / c), rho)
+ *   arena           DEVICE scratch owned by the caller, 256-byte aligned, at least spf_compress_host_arena_bytes(...)
+ *                   bytes; holds the device copies of the inputs, every intermediate and the scoring workspace
+ *   out_ids_host, out_pos_host (may be NULL)   HOST int32 [min(k * c, N)]
+ *   out_tok_spans_host, out_char_spans_host     HOST int32 [k][2]
+ *   out_counts_host                             HOST int64 [2]: {n_kept, n_spans}; only that many rows are written
+ *
+ * If the fused scoring kernel reports SPF_ERR_RANGE or SPF_ERR_TIMEOUT the prompt is scored again with the general
+ * kernels before anything is returned.  Errors: as the four calls; SPF_ERR_WORKSPACE for a small or misaligned arena;
+ * a device-side status that survives the retry is returned as the call's status.
+ */
+typedef struct {
+  int32_t chunk;        /* c >= 1                       */
+  int32_t pool_kernel;  /* w, odd, 1..255               */
+  double keep_ratio;    /* rho in (0, 1]                */
+} spf_select_params;
+
+SPF_API size_t spf_compress_host_arena_bytes(const spf_shape* shape, int64_t n_tokens, const spf_select_params* params);
+SPF_API int32_t spf_compress_host(const spf_shape* shape, int64_t n_tokens, const void* const* k_layers_host, const void* q_host,
+                                  const int32_t* token_ids_host, const int32_t* char_start_host, const int32_t* char_end_host,
+                                  const spf_select_params* params, void* arena, size_t arena_bytes, int32_t* out_ids_host,
+                                  int32_t* out_pos_host, int32_t* out_tok_spans_host, int32_t* out_char_spans_host,
+                                  int64_t* out_counts_host, void* cuda_stream);
 
 /*
  * Host helper for the keep rate of Section 3.1: the number of chunks a keep rate rho retains,

@@ -34,6 +34,10 @@ class _Prompt(ctypes.Structure):
                 ("importance", ctypes.c_void_p), ("lse", ctypes.c_void_p)]
 
 
+class _SelectParams(ctypes.Structure):
+    _fields_ = [("chunk", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("keep_ratio", ctypes.c_double)]
+
+
 class _PagedPrompt(ctypes.Structure):
     _fields_ = [("n_tokens", ctypes.c_int64), ("k_pools", ctypes.POINTER(ctypes.c_void_p)),
                 ("n_pool_blocks", ctypes.c_int64), ("block_tokens", ctypes.c_int32), ("block_table", ctypes.c_void_p),
@@ -76,6 +80,11 @@ def _load() -> ctypes.CDLL:
     dll.spf_select_topk_forced.argtypes = [vp, i64, i64, i32, i32, vp, vp]
     dll.spf_compact_spans.restype = i32
     dll.spf_compact_spans.argtypes = [vp, i64, i32, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    dll.spf_compress_host_arena_bytes.restype = ctypes.c_size_t
+    dll.spf_compress_host_arena_bytes.argtypes = [ctypes.POINTER(_Shape), i64, ctypes.POINTER(_SelectParams)]
+    dll.spf_compress_host.restype = i32
+    dll.spf_compress_host.argtypes = [ctypes.POINTER(_Shape), i64, ctypes.POINTER(ctypes.c_void_p), vp, vp, vp, vp,
+                                      ctypes.POINTER(_SelectParams), vp, ctypes.c_size_t, vp, vp, vp, vp, vp, vp]
     dll.spf_keep_count.restype = i64
     dll.spf_keep_count.argtypes = [i64, ctypes.c_double]
     dll.spf_keep_rate.restype = ctypes.c_double
@@ -396,6 +405,60 @@ def spf_compact_spans(kept_chunks: torch.Tensor, k: int, chunk: int, n_tokens: i
                                  _stream_ptr(stream)), "spf_compact_spans")
 
 
+def _host(t: torch.Tensor, dtype: torch.dtype, name: str) -> torch.Tensor:
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous host tensor of dtype {dtype}")
+    return t
+
+
+def spf_compress_host_arena_bytes(n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n_lookahead: int,
+                                  n_tokens: int, chunk: int, pool_kernel: int, keep: float, softmax_scale: float = 0.0) -> int:
+    shape = _Shape(n_layers, n_q_heads, n_kv_heads, head_dim, n_lookahead, float(softmax_scale))
+    prm = _SelectParams(chunk, pool_kernel, float(keep))
+    n = int(lib.spf_compress_host_arena_bytes(ctypes.byref(shape), n_tokens, ctypes.byref(prm)))
+    if n == 0:
+        raise SpfError(-1, "spf_compress_host_arena_bytes", spf_last_error())
+    return n
+
+
+def spf_compress_host(q: torch.Tensor, k_layers: Sequence[torch.Tensor], token_ids: torch.Tensor, char_start: torch.Tensor,
+                      char_end: torch.Tensor, chunk: int, pool_kernel: int, keep: float, arena: torch.Tensor,
+                      out_ids: torch.Tensor, out_pos: Optional[torch.Tensor], out_tok_spans: torch.Tensor,
+                      out_char_spans: torch.Tensor, out_counts: torch.Tensor, softmax_scale: float = 0.0,
+                      stream: Optional[torch.cuda.Stream] = None) -> None:
+    """The whole path for one prompt in HOST tensors (inputs and outputs); ``arena`` is device scratch.  Synchronises the
+    stream.  See spf_compress_host in include/spf.h for sizes."""
+    L, Hq, m, d = q.shape
+    Hkv, n, _ = k_layers[0].shape
+    _host(q, torch.bfloat16, "q")
+    for kl in k_layers:
+        _host(kl, torch.bfloat16, "k_layers[l]")
+        if tuple(kl.shape) != (Hkv, n, d):
+            raise ValueError("every k_layers[l] must be [Hkv, N, d]")
+    for name, t in (("token_ids", token_ids), ("char_start", char_start), ("char_end", char_end), ("out_ids", out_ids),
+                    ("out_tok_spans", out_tok_spans), ("out_char_spans", out_char_spans)):
+        _host(t, torch.int32, name)
+    if out_pos is not None:
+        _host(out_pos, torch.int32, "out_pos")
+    _host(out_counts, torch.int64, "out_counts")
+    if not arena.is_cuda:
+        raise TypeError("arena must be a CUDA tensor")
+    k = spf_keep_count((n + chunk - 1) // chunk, keep)
+    need = min(k * chunk, n)
+    if len(k_layers) != L or min(token_ids.numel(), char_start.numel(), char_end.numel()) < n or out_ids.numel() < need or \
+            (out_pos is not None and out_pos.numel() < need) or out_tok_spans.numel() < 2 * k or \
+            out_char_spans.numel() < 2 * k or out_counts.numel() < 2:
+        raise ValueError("a buffer is smaller than include/spf.h requires")
+    shape = _Shape(L, Hq, Hkv, d, m, float(softmax_scale))
+    prm = _SelectParams(chunk, pool_kernel, float(keep))
+    ptrs = (ctypes.c_void_p * L)(*[kl.data_ptr() for kl in k_layers])
+    _check(lib.spf_compress_host(ctypes.byref(shape), n, ctypes.cast(ptrs, ctypes.POINTER(ctypes.c_void_p)), q.data_ptr(),
+                                 token_ids.data_ptr(), char_start.data_ptr(), char_end.data_ptr(), ctypes.byref(prm),
+                                 arena.data_ptr(), arena.numel() * arena.element_size(), out_ids.data_ptr(), _ptr(out_pos),
+                                 out_tok_spans.data_ptr(), out_char_spans.data_ptr(), out_counts.data_ptr(),
+                                 _stream_ptr(stream)), "spf_compress_host")
+
+
 @dataclasses.dataclass
 class Selection:
     """Device-side result of one prompt; ``n_kept`` / ``n_spans`` are read from ``counts`` on demand."""
@@ -459,7 +522,9 @@ class Selector:
     def run(self, q: torch.Tensor, k_layers: Sequence[torch.Tensor], token_ids: torch.Tensor,
             char_start: torch.Tensor, char_end: torch.Tensor, keep: float,
             stream: Optional[torch.cuda.Stream] = None) -> Selection:
-        """Enqueues the whole path for one prompt whose tensors are already on the device."""
+        """Enqueues the whole path for one prompt whose tensors are already on the device.  Nothing is synchronised:
+        device-side conditions (see spf_score) accumulate in ``self.dev_status``, which the caller zeroes and reads
+        (run_checked does both)."""
         n = k_layers[0].shape[1]
         if n > self.max_tokens:
             raise ValueError(f"prompt has {n} tokens, selector was sized for {self.max_tokens}")
@@ -502,22 +567,33 @@ class Selector:
         return Selection(self.importance[:n], self.lse.view(L, Hq, m), self.chunk_scores[:n_chunks], k, self.kept,
                          self.out_ids, self.out_pos, self.tok_spans, self.char_spans, self.counts)
 
+    # device conditions after which the general path is tried: a row sum beyond fp32 (-6), a bounded wait that ran
+    # out (-5); and the host refusal of a grid that cannot be co-resident (-2, raised as SpfError)
+    _RETRY_ON = (-5, -6)
+
     def run_checked(self, q: torch.Tensor, k_layers: Sequence[torch.Tensor], token_ids: torch.Tensor,
                     char_start: torch.Tensor, char_end: torch.Tensor, keep: float,
                     stream: Optional[torch.cuda.Stream] = None) -> Selection:
         """Like run(), but synchronises and reads the device status.  If the fused scoring kernel reported
-        SPF_ERR_RANGE (a logit beyond its fp32 guard), the prompt is scored again on the general path, which
-        has no such limit.  Any other device status raises."""
+        SPF_ERR_RANGE (a row sum beyond fp32) or SPF_ERR_TIMEOUT (a bounded wait ran out, e.g. because its CTAs
+        could not all run at once), or refused the launch as unsupported, the prompt is scored again on the
+        general path, which has neither limit.  Any other status raises."""
+        s = stream or torch.cuda.current_stream()
         self.dev_status.zero_()
-        sel = self.run(q, k_layers, token_ids, char_start, char_end, keep, stream)
-        (stream or torch.cuda.current_stream()).synchronize()
-        status = int(self.dev_status.item())
-        if status == -6:
+        try:
+            sel = self.run(q, k_layers, token_ids, char_start, char_end, keep, stream)
+            s.synchronize()
+            status = int(self.dev_status.item())
+        except SpfError as err:
+            if err.status != -2:
+                raise
+            status = -2
+        if status in self._RETRY_ON or status == -2:
             previous = spf_set_score_path(1)
             try:
                 self.dev_status.zero_()
                 sel = self.run(q, k_layers, token_ids, char_start, char_end, keep, stream)
-                (stream or torch.cuda.current_stream()).synchronize()
+                s.synchronize()
                 status = int(self.dev_status.item())
             finally:
                 spf_set_score_path(previous)
@@ -527,16 +603,28 @@ class Selector:
 
     def run_host(self, q: torch.Tensor, k_layers: Sequence[torch.Tensor], token_ids: torch.Tensor,
                  char_start: torch.Tensor, char_end: torch.Tensor, keep: float):
-        """Same path for HOST tensors (ideally pinned): copies in, runs, copies the selection back.
+        """Same path for HOST tensors (ideally pinned) through spf_compress_host: one C call that copies in, runs and
+        copies the selection back.  The device arena and the pinned result buffers are kept between calls.
 
         Returns host NumPy arrays: kept ids, positions, token spans, character spans.
         """
-        dev = self.device
-        qd = q.to(dev, non_blocking=True)
-        kd = [t.to(dev, non_blocking=True) for t in k_layers]
-        idd, csd, ced = (t.to(dev, non_blocking=True) for t in (token_ids, char_start, char_end))
-        sel = self.run(qd, kd, idd, csd, ced, keep)
-        counts = sel.counts.cpu()
+        L, Hq, Hkv, d, m = self.geom
+        n = k_layers[0].shape[1]
+        need = spf_compress_host_arena_bytes(L, Hq, Hkv, d, m, n, self.chunk, self.pool_kernel, keep, self.softmax_scale)
+        if getattr(self, "_arena", None) is None or self._arena.numel() < need:
+            self._arena = torch.empty(need, dtype=torch.uint8, device=self.device)
+        k = spf_keep_count((n + self.chunk - 1) // self.chunk, keep)
+        rows = min(k * self.chunk, n)
+        host = getattr(self, "_host_out", None)
+        if host is None or host[0].numel() < rows or host[2].numel() < 2 * k:
+            host = [torch.empty(rows, dtype=torch.int32).pin_memory(), torch.empty(rows, dtype=torch.int32).pin_memory(),
+                    torch.empty((k, 2), dtype=torch.int32).pin_memory(), torch.empty((k, 2), dtype=torch.int32).pin_memory(),
+                    torch.empty(2, dtype=torch.int64).pin_memory()]
+            self._host_out = host
+        ids, pos, tok, ch, counts = host
+        with torch.cuda.device(self.device):
+            spf_compress_host(q, k_layers, token_ids, char_start, char_end, self.chunk, self.pool_kernel, keep, self._arena,
+                              ids, pos, tok, ch, counts, self.softmax_scale)
         n_kept, n_spans = int(counts[0]), int(counts[1])
-        return dict(ids=sel.out_ids[:n_kept].cpu().numpy(), pos=sel.out_pos[:n_kept].cpu().numpy(),
-                    tok_spans=sel.tok_spans[:n_spans].cpu().numpy(), char_spans=sel.char_spans[:n_spans].cpu().numpy())
+        return dict(ids=ids[:n_kept].numpy().copy(), pos=pos[:n_kept].numpy().copy(), tok_spans=tok[:n_spans].numpy().copy(),
+                    char_spans=ch[:n_spans].numpy().copy())

@@ -116,7 +116,7 @@ extern "C" size_t spf_score_workspace_bytes(const spf_shape* shape, const spf_pr
 }
 
 static int32_t score_impl(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, const float* const* extra_lse,
-                          void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+                          void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream, int path_override = -1) {
   clear_error();
   if (shape == nullptr || prompts == nullptr || n_prompts < 1)
     return fail(SPF_ERR_INVALID_ARG, "spf_score: null argument or n_prompts < 1");
@@ -142,7 +142,7 @@ static int32_t score_impl(const spf_shape* shape, const spf_prompt* prompts, int
     ScoreProblem p;
     make_problem(shape, prompts[i], i, &p);
     if (extra_lse != nullptr) p.extra_lse = extra_lse[i];
-    const int path = g_score_path.load(std::memory_order_relaxed);
+    const int path = path_override >= 0 ? path_override : g_score_path.load(std::memory_order_relaxed);
     const bool fused = path == 2 || (path == 0 && score_fused_supported(p, sm_count));
     const int32_t st = fused ? score_fused_launch(p, workspace, sm_count, dev_status, stream)
                              : score_mma_launch(p, workspace, sm_count, stream);
@@ -150,6 +150,13 @@ static int32_t score_impl(const spf_shape* shape, const spf_prompt* prompts, int
   }
   return SPF_OK;
 }
+
+namespace spf {
+int32_t score_on_path(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace, size_t workspace_bytes,
+                      int32_t* dev_status, void* cuda_stream, int path) {
+  return score_impl(shape, prompts, n_prompts, nullptr, workspace, workspace_bytes, dev_status, cuda_stream, path);
+}
+}  // namespace spf
 
 extern "C" int32_t spf_score(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace,
                              size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {

@@ -41,6 +41,10 @@ bool score_fused_supported(const ScoreProblem& p, int sm_count);
 size_t score_fused_workspace_bytes(const ScoreProblem& p);
 int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count, int32_t* dev_status, cudaStream_t stream);
 
+// spf_score with the kernel path given for this call only (0 automatic, 1 general, 2 fused) instead of the process-wide setting.
+int32_t score_on_path(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace, size_t workspace_bytes,
+                      int32_t* dev_status, void* cuda_stream, int path);
+
 // Launches the one-CTA self-test of the kernels' bounded wait (see spf_selftest_bounded_wait).
 int32_t bounded_wait_selftest_launch(int32_t* dev_status, cudaStream_t stream);
 

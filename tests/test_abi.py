@@ -102,3 +102,21 @@ def test_score_shape_validation(spf):
     arr = (_Prompt * 1)(good)
     assert lib.spf_score_workspace_bytes(ctypes.byref(_Shape(2, 4, 2, 64, 8, 0.0)), arr, 1) > 0
     assert lib.spf_score_workspace_bytes(ctypes.byref(_Shape(2, 4, 2, 96, 8, 0.0)), arr, 1) == 0
+
+
+def test_compress_host_validates_before_touching_the_device(spf):
+    """Host-side checks of spf_compress_host: arena size query, null pointers, small arena (nothing is launched)."""
+    from paper_2603_02631_b200.binding import _SelectParams, _Shape
+    shape = _Shape(2, 4, 2, 64, 8, 0.0)
+    prm = _SelectParams(32, 13, 0.25)
+    need = spf.lib.spf_compress_host_arena_bytes(ctypes.byref(shape), 1000, ctypes.byref(prm))
+    # the arena holds at least the device copy of the key cache, queries, ids and offsets
+    assert need >= 2 * 2 * 1000 * 64 * 2 + 2 * 4 * 8 * 64 * 2 + 3 * 4 * 1000
+    assert spf.lib.spf_compress_host_arena_bytes(None, 1000, ctypes.byref(prm)) == 0
+    assert spf.lib.spf_compress_host_arena_bytes(ctypes.byref(shape), 0, ctypes.byref(prm)) == 0
+    bad = _Shape(2, 4, 2, 96, 8, 0.0)                       # head_dim 96 is outside the kernels
+    assert spf.lib.spf_compress_host_arena_bytes(ctypes.byref(bad), 1000, ctypes.byref(prm)) == 0
+    none = ctypes.c_void_p(None)
+    rc = spf.lib.spf_compress_host(ctypes.byref(shape), 1000, None, none, none, none, none, ctypes.byref(prm), none, 0,
+                                   none, none, none, none, none, none)
+    assert rc == -1

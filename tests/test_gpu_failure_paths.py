@@ -69,3 +69,71 @@ def test_selector_checked_run_falls_back_to_the_general_path():
     want, _ = oracle.token_importance(bf16_bits(q), [bf16_bits(x) for x in k])
     assert_importance_close(res.importance.cpu().numpy(), want)
     assert 0 in res.kept_chunks[:res.k].cpu().tolist()     # the dominant key 7 lives in chunk 0
+
+
+def _offset_case(offsets_nats, seed=5, n=3000):
+    """One kv-head with a group of four query heads whose logits carry constant offsets (in nats): every key has
+    16 in coordinate 0 and head g has offsets[g] / 2 there, so head g's logits are shifted by offsets[g] (scale
+    1/8).  The softmax does not see a constant shift; a per-slab reference does."""
+    L, Hq, Hkv, d, m = 2, 4, 1, 64, 8
+    g = torch.Generator().manual_seed(seed)
+    q = torch.randn(L, Hq, m, d, generator=g)
+    k = [torch.randn(Hkv, n, d, generator=g) for _ in range(L)]
+    for layer in range(L):
+        k[layer][..., 0] = 16.0
+        for h, off in enumerate(offsets_nats):
+            q[layer, h, :, 0] = off / 2.0
+    return q.to(torch.bfloat16), [x.to(torch.bfloat16) for x in k]
+
+
+def _score(spf, q, k, path):
+    n = k[0].shape[1]
+    previous = spf.spf_set_score_path(path)
+    try:
+        imp = torch.zeros(n, dtype=torch.float32, device="cuda")
+        lse = torch.zeros(q.shape[0] * q.shape[1] * q.shape[2], dtype=torch.float32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        bufs = spf.PromptBuffers(q.cuda(), [x.cuda() for x in k], imp, lse)
+        ws = torch.empty(spf.spf_score_workspace_bytes([bufs]), dtype=torch.uint8, device="cuda")
+        spf.spf_score([bufs], ws, 0.0, status)
+        torch.cuda.synchronize()
+        return int(status.item()), imp.cpu().numpy(), lse.cpu().numpy()
+    finally:
+        spf.spf_set_score_path(previous)
+
+
+@pytest.mark.parametrize("offsets", [(0.0, -30.0, -45.0, 10.0), (0.0, -70.0, 20.0, -80.0), (60.0, 0.0, 0.0, 0.0)])
+def test_fused_path_is_exact_when_heads_of_a_group_differ_in_scale(offsets):
+    """Heads that share a kv-head, tens of nats apart: the fused path's single reference per kv-head must not cost
+    the low heads any part of their row sums (importance and lse against the oracle, status 0)."""
+    import paper_2603_02631_b200 as spf
+    q, k = _offset_case(offsets)
+    want, want_lse = oracle.token_importance(bf16_bits(q), [bf16_bits(x) for x in k])
+    status, imp, lse = _score(spf, q, k, 2)
+    assert status == 0
+    assert_importance_close(imp, want)
+    # logits reach 80 nats here: fp32 spacing there is 8e-6, the accumulated error a few 1e-4
+    np.testing.assert_allclose(lse.reshape(want_lse.shape), want_lse, rtol=0, atol=1e-3)
+
+
+def test_fused_path_range_limit_is_on_the_high_side_only():
+    """A head 150 nats (216 base-2 units) above the lowest head of its group overflows the fp32 row sums of the
+    fused path: status SPF_ERR_RANGE, nothing else; 80 nats below is fine (previous test).  The checked run
+    recovers on the general path and matches the oracle."""
+    import paper_2603_02631_b200 as spf
+    q, k = _offset_case((0.0, 150.0, 0.0, 0.0))
+    want, _ = oracle.token_importance(bf16_bits(q), [bf16_bits(x) for x in k])
+    status, _, _ = _score(spf, q, k, 2)
+    assert status == -6
+    status, imp, _ = _score(spf, q, k, 1)
+    assert status == 0
+    assert_importance_close(imp, want)
+    n = k[0].shape[1]
+    sel = spf.Selector(2, 4, 1, 64, 8, max_tokens=n, chunk=32)
+    ids = torch.arange(n, dtype=torch.int32, device="cuda")
+    previous = spf.spf_set_score_path(2)
+    try:
+        res = sel.run_checked(q.cuda(), [x.cuda() for x in k], ids, ids * 2, ids * 2 + 2, keep=0.1)
+    finally:
+        spf.spf_set_score_path(previous)
+    assert_importance_close(res.importance.cpu().numpy(), want)

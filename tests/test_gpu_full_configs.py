@@ -1,7 +1,8 @@
 """Parity at the full sizes of the five workload configurations, in the launch configuration bench.py times.
 
 Inputs are generated on the GPU and the same bytes are copied to the host for the oracle.  Both scoring paths
-(fused single kernel, general two-sweep) are checked against one oracle run per prompt.
+(fused single kernel, general two-sweep) are checked against one oracle run per prompt; of the ragged batch every
+prompt is checked on the fused path (the one the bench times), the shortest and the longest on both.
 """
 import numpy as np
 import pytest
@@ -18,15 +19,20 @@ CASES = [
     ("small32k", [0]),
     ("wide64k", [0]),
     ("long128k", [0]),
-    ("ragged8", None),      # the shortest and the longest prompt of the batch (filled in below)
+    ("ragged8", None),      # all prompts of the batch
 ]
 
 
 def _prompt_indices(name, idx):
-    if idx is not None:
-        return idx
+    return idx if idx is not None else list(range(len(CONFIGS[name].lengths)))
+
+
+def _paths(name, index):
+    """Kernel paths to check for this prompt: both, except the middle prompts of the ragged batch (fused only)."""
     lengths = CONFIGS[name].lengths
-    return sorted({int(np.argmin(lengths)), int(np.argmax(lengths))})
+    if len(lengths) == 1 or index in (int(np.argmin(lengths)), int(np.argmax(lengths))):
+        return (2, 1)
+    return (2,)
 
 
 @pytest.mark.parametrize("name,idx", CASES)
@@ -44,7 +50,7 @@ def test_full_size_config(name, idx):
         want_scores = oracle.chunk_means(oracle.avg_pool(want_imp, cfg.pool_kernel), cfg.chunk)
         sel = spf.Selector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, n,
                            chunk=cfg.chunk, pool_kernel=cfg.pool_kernel)
-        for path in (2, 1):
+        for path in _paths(name, index):
             previous = spf.spf_set_score_path(path)
             try:
                 for keep in cfg.keep:

@@ -3,8 +3,10 @@
 A serving engine that has handed all free HBM to its KV-cache pool, or code that must not trigger
 the device-wide synchronisation of cudaMalloc, cannot provide the workspace spf_score asks for.
 spf_score_static uses a fixed scratch array inside the library instead.  These tests call it through
-the C ABI and require the same importance and log-sum-exp as spf_score gives with a caller-owned
-workspace, on two calls in a row (the second one sees whatever the first left in the shared array).
+the C ABI and require the importance and log-sum-exp of the CPU oracle, and of spf_score with a caller-owned
+workspace, on two calls in a row (the second one sees whatever the first left in the shared array); and they
+require that the call leaves the amount of free device memory exactly as it found it, which is the property the
+entry point exists for.
 
 This file is named so that pytest collects it last.
 """
@@ -14,9 +16,10 @@ import numpy as np
 import pytest
 import torch
 
-from workloads import make_prompt, small_config
+import oracle
+from workloads import bf16_bits, make_prompt, small_config
 
-from parity_util import IMPORTANCE_RTOL
+from parity_util import IMPORTANCE_RTOL, assert_importance_close
 
 
 def _score_both(spf, prompt):
@@ -31,7 +34,16 @@ def _score_both(spf, prompt):
         lse = torch.full((n_rows,), float("nan"), dtype=torch.float32, device="cuda")
         bufs = spf.PromptBuffers(dp.q, dp.k, imp, lse)
         if static:
+            # everything the call touches is allocated by now; the call itself must not change what the device has free
+            # (measured at the driver, below torch's caching allocator) nor what torch has handed out
+            torch.cuda.synchronize()
+            free_before, _ = torch.cuda.mem_get_info()
+            torch_before = torch.cuda.memory_allocated()
             spf.spf_score_static([bufs])
+            torch.cuda.synchronize()
+            free_after, _ = torch.cuda.mem_get_info()
+            assert free_after == free_before, f"spf_score_static changed free device memory by {free_before - free_after} bytes"
+            assert torch.cuda.memory_allocated() == torch_before
         else:
             ws = torch.empty(spf.spf_score_workspace_bytes([bufs]), dtype=torch.uint8, device="cuda")
             spf.spf_score([bufs], ws)
@@ -49,9 +61,18 @@ def test_static_scratch_matches_workspace_path_twice_in_a_row():
         small_config("noalloc_a", n_layers=4, n_q_heads=8, n_kv_heads=2, head_dim=64, n_lookahead=16, lengths=(6001,), seed=31),
         small_config("noalloc_b", n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=128, n_lookahead=8, lengths=(1500,), seed=32),
     ]
+    # the first call on a device looks the scratch array up (and loads the module that holds it): done here, outside
+    # the calls whose memory footprint is checked
+    warm = make_prompt(small_config("noalloc_warm", n_layers=1, n_q_heads=2, n_kv_heads=1, head_dim=64, n_lookahead=8,
+                                    lengths=(200,), seed=30)).to("cuda")
+    spf.spf_score_static([spf.PromptBuffers(warm.q, warm.k, torch.empty(200, dtype=torch.float32, device="cuda"), None)])
+    torch.cuda.synchronize()
     for cfg in shapes:
         prompt = make_prompt(cfg)
         (imp_ws, lse_ws), (imp_st, lse_st) = _score_both(spf, prompt)
+        want_imp, want_lse = oracle.token_importance(bf16_bits(prompt.q), [bf16_bits(x) for x in prompt.k])
+        assert_importance_close(imp_st, want_imp)
+        np.testing.assert_allclose(lse_st, want_lse.reshape(-1), rtol=0, atol=2e-4)
         assert np.isfinite(imp_st).all() and np.isfinite(lse_st).all()
         rel = np.abs(imp_st - imp_ws) / np.maximum(np.abs(imp_ws), 1e-30)
         assert rel.max() <= IMPORTANCE_RTOL, f"{cfg.name}: importance differs by {rel.max():.3e}"

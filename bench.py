@@ -62,6 +62,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--sustained-seconds", type=float, default=1.5,
+                    help="length of the back-to-back spf_score loop behind the `sustained` record (0: skip)")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the scoring fractions of the other workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--score-path", default="auto", choices=["auto", "general", "fused"],
                     help="kernels behind spf_score: fused single-kernel path, general two-sweep path, or automatic")
@@ -79,9 +82,11 @@ def hbm_peak():
 
 # ----------------------------------------------------------------------------------------------- clocks
 class ClockSampler:
+    """nvidia-smi polled every 10 ms into a file; mark() remembers a position, stats(lo, hi) summarises a span."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index: int):
         self.index = index
@@ -89,50 +94,72 @@ class ClockSampler:
         self.path = None
 
     def start(self):
-        """Starts nvidia-smi sampling every 50 ms and waits (up to 5 s) for its first line."""
+        """Starts the sampling and waits (up to 5 s) for its first line."""
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "10",
                  "-i", str(self.index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
             deadline = time.time() + 5.0
             while time.time() < deadline and os.path.getsize(self.path) == 0:
                 time.sleep(0.02)
-            self.skip = sum(1 for _ in open(self.path))      # lines written before the timed region
         except Exception:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def mark(self) -> int:
+        """Number of samples written so far."""
         if self.proc is None:
-            return out
+            return 0
+        try:
+            return sum(1 for _ in open(self.path))
+        except OSError:
+            return 0
+
+    def stop(self):
+        if self.proc is None:
+            return
+        time.sleep(0.03)                                   # let the sample that covers the last launches land
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+
+    def stats(self, lo: int = 0, hi: int = None):
+        """Median SM clock, maximum clock and the throttle reasons seen in samples lo..hi (one before lo is included:
+        it covers the start of the span)."""
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "power_w": None}
+        if self.path is None:
+            return out
+        sm, mx, pw, reasons = [], [], [], set()
         try:
-            for line in list(open(self.path))[getattr(self, "skip", 0):]:
-                parts = [p.strip() for p in line.split(",")]
-                if len(parts) < 7:
-                    continue
-                try:
-                    sm.append(float(parts[0]))
-                    mx.append(float(parts[1]))
-                except ValueError:
-                    continue
-                for name, val in zip(names, parts[3:7]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
+            lines = list(open(self.path))
+        except OSError:
+            return out
+        for line in lines[max(lo - 1, 0):hi]:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(self.NAMES, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm),
+                       power_w=statistics.median(pw))
+        return out
+
+    def close(self):
+        try:
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
-        return out
 
 
 # ----------------------------------------------------------------------------------------------- oracle leg
@@ -233,6 +260,52 @@ def whole_job_value(tokens_per_rank_step, steps, world, ms_total_max):
 
 
 # ----------------------------------------------------------------------------------------------- our arm
+def score_bytes(cfg):
+    """Algorithmic bytes of one spf_score pass over the workload: K read once, Q, importance and lse written."""
+    n_prompts = len(cfg.lengths)
+    rows = cfg.n_layers * cfg.n_q_heads * cfg.n_lookahead
+    return cfg.k_bytes() + n_prompts * rows * cfg.head_dim * 2 + 4 * sum(cfg.lengths) + n_prompts * rows * 4
+
+
+def time_score_launches(spf, sel, prompts, launches, stream):
+    """Average CUDA-event duration of `launches` passes of spf_score over `prompts` (one event pair around all)."""
+    import torch
+    bufs = [spf.binding.PromptBuffers(p.q, p.k, sel.importance[:p.n_tokens], sel.lse) for p in prompts]
+    ws = sel._workspace(max(bufs, key=lambda b: b.importance.numel()))
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(launches):
+        for bf in bufs:
+            spf.spf_score([bf], ws, 0.0, sel.dev_status)
+    b.record(stream)
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / launches
+
+
+def secondary_workloads(spf, dev, peak, stream, names=("small32k", "wide64k", "ragged8")):
+    """Scoring fraction of the HBM rate on the other workload configurations (20 launches each after 3 warm-ups)."""
+    import torch
+    from workloads import CONFIGS, make_prompt
+    out = []
+    for name in names:
+        cfg = CONFIGS[name]
+        try:
+            prompts = [make_prompt(cfg, i, dev) for i in range(len(cfg.lengths))]
+            sel = spf.Selector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, max(cfg.lengths),
+                               chunk=cfg.chunk, pool_kernel=cfg.pool_kernel, device=dev)
+            time_score_launches(spf, sel, prompts, 3, stream)
+            ms = time_score_launches(spf, sel, prompts, 20, stream)
+            status = int(sel.dev_status.item())
+            gbs = score_bytes(cfg) / (ms * 1e-3) / 1e9
+            out.append({"workload": name, "ms_per_launch": ms, "achieved": gbs, "frac": gbs / peak, "dev_status": status,
+                        "tokens": sum(cfg.lengths)})
+            del prompts, sel
+            torch.cuda.empty_cache()
+        except Exception as err:                           # e.g. not enough free memory for the 36 GB batch
+            out.append({"workload": name, "error": str(err)[:200]})
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -294,19 +367,18 @@ def run_ours(args):
     sampler.start()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    m0 = sampler.mark()
     t_start.record(stream)
     for _ in range(args.steps):
         step()
     t_end.record(stream)
     barrier()
-    clocks = sampler.stop()
     ms_total = t_start.elapsed_time(t_end)
     status = int(sel.dev_status.item())
     if status != 0:
         raise RuntimeError(f"device status {status} ({spf.spf_status_string(status)}) after the timed region")
 
     # --- the scoring call on its own (same launches, events around spf_score only) --------------------
-    score_ms = []
     bufs = [spf.binding.PromptBuffers(p.q, p.k, sel.importance[:p.n_tokens], sel.lse) for p in prompts]
     ws = sel._workspace(bufs[cfg.lengths.index(max_n)])
     events = []
@@ -318,10 +390,27 @@ def run_ours(args):
         b.record(stream)
         events.append((a, b))
     torch.cuda.synchronize()
+    m1 = sampler.mark()
     score_ms = [a.elapsed_time(b) for a, b in events]
     score_ms_avg = sum(score_ms) / len(score_ms)
 
-    # --- end to end from pinned host memory -----------------------------------------------------
+    # --- sustained: the scoring call back to back for a second or more (the power-capped steady state) ------------
+    sustained = None
+    if args.sustained_seconds > 0:
+        launches = max(10, int(args.sustained_seconds * 1e3 / score_ms_avg))
+        m2 = sampler.mark()
+        ms = time_score_launches(spf, sel, prompts, launches, stream)
+        m3 = sampler.mark()
+        sustained = {"launches": launches, "ms_per_launch": ms}
+    sampler.stop()
+    clocks = sampler.stats(m0, m1)
+    if sustained:
+        c = sampler.stats(m2, m3)
+        sustained.update(sm_mhz=c["sm_mhz"], power_w=c["power_w"], reasons=c["reasons"], samples=c["samples"],
+                         ms_x_mhz=(sustained["ms_per_launch"] * c["sm_mhz"]) if c["sm_mhz"] else None)
+    sampler.close()
+
+    # --- end to end: host buffers through the C entry point spf_compress_host ---------------------------------------
     e2e = None
     if args.e2e_steps > 0:
         host = []
@@ -339,7 +428,7 @@ def run_ours(args):
             d2h = 0
             for hp in host:
                 out = sel.run_host(hp["q"], hp["k"], hp["ids"], hp["cs"], hp["ce"], keep)
-                d2h += 16 + sum(v.nbytes for v in out.values())
+                d2h += 16 + 4 + sum(v.nbytes for v in out.values())
             return d2h
 
         e2e_step()
@@ -351,6 +440,9 @@ def run_ours(args):
         barrier()
         e2e_s = time.perf_counter() - t0
         e2e = {"seconds": e2e_s, "h2d": h2d, "d2h": d2h}
+        del host
+        sel._arena = None
+        torch.cuda.empty_cache()
 
     # --- reduce over ranks --------------------------------------------------------------------------
     ms_total, e2e_s_max, score_ms_avg = max_over_ranks([ms_total, e2e["seconds"] if e2e else 0.0, score_ms_avg], dev, world)
@@ -364,9 +456,8 @@ def run_ours(args):
     value = whole_job_value(tokens_per_step, args.steps, world, ms_total)
     peak, peak_kind = hbm_peak()
     k_bytes = cfg.k_bytes()
-    q_bytes = n_prompts * cfg.n_layers * cfg.n_q_heads * cfg.n_lookahead * cfg.head_dim * 2
-    score_bytes = k_bytes + q_bytes + 4 * tokens_per_step + n_prompts * cfg.n_layers * cfg.n_q_heads * cfg.n_lookahead * 4
-    achieved = score_bytes / (score_ms_avg * 1e-3) / 1e9
+    sbytes = score_bytes(cfg)
+    achieved = sbytes / (score_ms_avg * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
@@ -377,16 +468,23 @@ def run_ours(args):
                    "pool_kernel": cfg.pool_kernel, "k_cache_bytes": k_bytes,
                    "l2": "inputs larger than L2 (key cache streamed every step)", "parallelism": f"prompts x{world}"},
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                   "samples": clocks["samples"]},
+                   "samples": clocks["samples"], "span": "timed steps + the spf_score-only launches, 10 ms period"},
         "gpu_launches": launches_per_prompt * n_prompts * args.steps,
         "roofline": {"bound": "hbm", "kernel": f"spf_score ({score_kernels})",
                      "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                      "frac": achieved / peak, "traffic": ncu_traffic(cfg.name, "fused" if fused else "general"), "ms_per_launch": score_ms_avg,
-                     "algorithmic_bytes": score_bytes},
+                     "algorithmic_bytes": sbytes},
     }
+    if sustained:
+        gbs = sbytes / (sustained["ms_per_launch"] * 1e-3) / 1e9
+        sustained.update(achieved=gbs, frac=gbs / peak)
+        line["sustained"] = sustained
     if e2e:
         line["e2e"] = {"value": world * tokens_per_step * args.e2e_steps / e2e["seconds"], "unit": UNIT,
-                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": args.e2e_steps}
+                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": args.e2e_steps,
+                       "api": "spf_compress_host (C ABI, pinned host buffers, device arena reused between calls)"}
+    if world == 1 and not args.no_secondary and cfg.name == DEFAULT_WORKLOAD:
+        line["secondary"] = secondary_workloads(spf, dev, peak, stream)
     if world == 1 and not args.no_cpu_baseline:
         cpu_prompt = make_prompt(cfg, 0, dev).to("cpu")
         v, secs, desc = oracle_sample(cfg, cpu_prompt, keep, pick_sample_layers(cfg, cpu_prompt))

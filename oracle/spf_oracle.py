@@ -43,6 +43,22 @@ def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
 
 
+def fp8_e4m3_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact value of 8-bit floating-point patterns (uint8) in the E4M3 format serving systems use for KV caches:
+    1 sign bit, 4 exponent bits (bias 7), 3 mantissa bits; exponent field 0 holds the subnormals m/8 * 2^-6; there are
+    no infinities, and exponent 15 with mantissa 7 is NaN (everything else with exponent 15 is an ordinary number,
+    up to 448).  Written out from the format's definition, bit field by bit field."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint8).astype(np.int64)
+    sign = np.where(bits & 0x80, -1.0, 1.0)
+    e = (bits >> 3) & 0xF
+    m = (bits & 0x7).astype(np.float64)
+    normal = (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64))
+    subnormal = (m / 8.0) * 2.0 ** -6
+    value = np.where(e == 0, subnormal, normal)
+    value = np.where((e == 15) & (bits & 0x7 == 7), np.nan, value)
+    return sign * value
+
+
 # --------------------------------------------------------------------------------------
 # Appendix A.1.1 -- attention-based token importance (Algorithm 1, AggregateMaxMean)
 # --------------------------------------------------------------------------------------
@@ -91,6 +107,35 @@ def token_importance(q_bits: np.ndarray, k_bits: Sequence[np.ndarray], scale: Op
                     whole = np.logaddexp(lse[l, h], np.asarray(extra_lse, dtype=np.float64)[l, h])
                     p = p * np.exp(lse[l, h] - whole)[:, None]      # the prompt's share of the larger denominator
                     lse[l, h] = whole
+                np.maximum(A, p, out=A)
+    return A.mean(axis=0), lse
+
+
+def token_importance_fp8(q_bits: np.ndarray, k_bytes: Sequence[np.ndarray], k_scale: np.ndarray,
+                         scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """token_importance for a key cache stored in 8 bits (Section 3.1: the serving system's KV caches; a draft
+    model served the same way keeps its keys quantised).  The cache format is an INPUT format: key (l, hk, s, j) has
+    the value k_scale[l, hk] * E4M3(k_bytes[l][hk, s, j]), decoded exactly; everything after that is Appendix A.1.1
+    unchanged.
+
+    q_bits: uint16 [L, Hq, m, d] (bf16 patterns); k_bytes: L arrays uint8 [Hkv, N, d]; k_scale: fp32 [L, Hkv].
+    Returns (I [N], lse [L, Hq, m]) in fp64.
+    """
+    L, Hq, m, d = q_bits.shape
+    Hkv, N, d2 = k_bytes[0].shape
+    assert d2 == d and len(k_bytes) == L and Hq % Hkv == 0
+    k_scale = np.asarray(k_scale, dtype=np.float32).astype(np.float64).reshape(L, Hkv)
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    A = np.zeros((m, N), dtype=np.float64)
+    lse = np.zeros((L, Hq, m), dtype=np.float64)
+    for l in range(L):
+        for hk in range(Hkv):
+            k_lh = k_scale[l, hk] * fp8_e4m3_to_f64(k_bytes[l][hk])
+            for g in range(G):
+                h = hk * G + g
+                p, lse[l, h] = softmax_rows(attention_logits(bf16_to_f64(q_bits[l, h]), k_lh, scale))
                 np.maximum(A, p, out=A)
     return A.mean(axis=0), lse
 

@@ -12,5 +12,6 @@ from .synthetic import (  # noqa: F401
     bf16_bits,
     make_prompt,
     make_workload,
+    quantize_keys_e4m3,
     small_config,
 )

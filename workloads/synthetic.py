@@ -137,6 +137,21 @@ def bf16_bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().contiguous().cpu().view(torch.int16).numpy().view(np.uint16)
 
 
+def quantize_keys_e4m3(k: Sequence[torch.Tensor]):
+    """An 8-bit copy of a bf16 key cache as a serving system would hold it: per (layer, kv-head) one fp32 scale
+    (largest magnitude / 448, the format's largest number) and the keys divided by it, rounded to E4M3 by torch.
+    Returns (L uint8 tensors [Hkv, N, d], fp32 scales [L, Hkv]).  Input preparation only: what the bytes MEAN is
+    defined by the consumer (scale * E4M3 value)."""
+    bytes_, scales = [], []
+    for kl in k:
+        amax = kl.float().abs().amax(dim=(1, 2)).clamp_min(1e-12)
+        sc = (amax / 448.0).to(torch.float32)
+        q8 = (kl.float() / sc[:, None, None]).to(torch.float8_e4m3fn)
+        bytes_.append(q8.view(torch.uint8).contiguous())
+        scales.append(sc)
+    return bytes_, torch.stack(scales).contiguous()
+
+
 def _place_needles(rng: np.random.Generator, n_tokens: int, cfg: WorkloadConfig):
     """Non-overlapping spans: one per equal segment of the prompt, uniform inside it."""
     count = cfg.n_needles

@@ -12,7 +12,8 @@
  *   spf_compact_spans  Section 3.2 / Algorithm 1 "MergeAdjacentChunks" + "MapDraftChunksToTextSpans".
  *
  * Around them: spf_keep_count / spf_keep_rate / spf_snap_budget (Section 3.1, keep rate) and spf_concat_with_delim
- * (Algorithm 1 "ConcatWithDelim") on the host; spf_score_paged (paged key cache), spf_score_shard_lse /
+ * (Algorithm 1 "ConcatWithDelim") on the host; spf_score_paged (paged key cache), spf_score_fp8 (8-bit key cache),
+ * spf_score_shard_lse /
  * spf_score_shard_apply (one prompt's keys over several GPUs); spf_score_extra, spf_chunk_pool_edge,
  * spf_select_topk_forced (switches for points the paper leaves open); spf_compress_host (the four calls for host
  * buffers); spf_score_static (no allocation).
@@ -170,6 +171,40 @@ typedef struct {
 SPF_API size_t spf_score_paged_workspace_bytes(const spf_shape* shape, const spf_paged_prompt* prompts, int32_t n_prompts);
 SPF_API int32_t spf_score_paged(const spf_shape* shape, const spf_paged_prompt* prompts, int32_t n_prompts, void* workspace,
                                 size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * spf_score on an 8-BIT key cache (Section 3.1: the paper's serving system keeps KV caches in block-quantised form; a
+ * draft model served the same way holds its prompt keys in 8 bits).  The cache format is an input format: key
+ * (l, hk, s, j) has the value
+ *     k_scale[l * Hkv + hk] * E4M3(byte at k_layers[l] + hk * k_stride_head + s * k_stride_tok + j)
+ * with E4M3 the 8-bit floating-point format of 1 sign, 4 exponent (bias 7) and 3 mantissa bits, subnormals, no
+ * infinities (the byte patterns 0x7F / 0xFF, NaN, must not occur).  Bytes are widened to bf16 exactly and the scale is
+ * folded into the softmax scale of its (layer, kv-head), so the arithmetic and its error are those of spf_score.
+ * Queries stay bf16.
+ *
+ *   k_layers       HOST array of L device pointers (8-byte aligned), layer l uint8 [Hkv][N][d]; strides in bytes,
+ *                  k_stride_tok >= d, both strides multiples of 8
+ *   k_scale        DEVICE fp32 [L][Hkv], positive and finite
+ *   others         as in spf_prompt
+ *
+ * Only the general two-sweep kernels read this format (they read the cache twice, so halving its bytes is where it
+ * pays); with the fused path forced (spf_set_score_path(2)) the call returns SPF_ERR_UNSUPPORTED.  `dev_status` is
+ * accepted for symmetry and never written.  Workspace: spf_score_fp8_workspace_bytes(...), rules as for spf_score.
+ */
+typedef struct {
+  int64_t n_tokens;
+  const void* const* k_layers;
+  int64_t k_stride_head;
+  int64_t k_stride_tok;
+  const float* k_scale;
+  const void* q;
+  float* importance;
+  float* lse;
+} spf_fp8_prompt;
+
+SPF_API size_t spf_score_fp8_workspace_bytes(const spf_shape* shape, const spf_fp8_prompt* prompts, int32_t n_prompts);
+SPF_API int32_t spf_score_fp8(const spf_shape* shape, const spf_fp8_prompt* prompts, int32_t n_prompts, void* workspace,
+                              size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
 
 /*
  * One long prompt over several GPUs (Appendix A.1.1 is per prompt; this shards its keys).  Each rank holds a contiguous

@@ -34,6 +34,12 @@ class _Prompt(ctypes.Structure):
                 ("importance", ctypes.c_void_p), ("lse", ctypes.c_void_p)]
 
 
+class _Fp8Prompt(ctypes.Structure):
+    _fields_ = [("n_tokens", ctypes.c_int64), ("k_layers", ctypes.POINTER(ctypes.c_void_p)),
+                ("k_stride_head", ctypes.c_int64), ("k_stride_tok", ctypes.c_int64), ("k_scale", ctypes.c_void_p),
+                ("q", ctypes.c_void_p), ("importance", ctypes.c_void_p), ("lse", ctypes.c_void_p)]
+
+
 class _SelectParams(ctypes.Structure):
     _fields_ = [("chunk", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("keep_ratio", ctypes.c_double)]
 
@@ -60,6 +66,10 @@ def _load() -> ctypes.CDLL:
     dll.spf_score_paged_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_PagedPrompt), i32]
     dll.spf_score_paged.restype = i32
     dll.spf_score_paged.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_PagedPrompt), i32, vp, ctypes.c_size_t, vp, vp]
+    dll.spf_score_fp8_workspace_bytes.restype = ctypes.c_size_t
+    dll.spf_score_fp8_workspace_bytes.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Fp8Prompt), i32]
+    dll.spf_score_fp8.restype = i32
+    dll.spf_score_fp8.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Fp8Prompt), i32, vp, ctypes.c_size_t, vp, vp]
     dll.spf_score_shard_lse.restype = i32
     dll.spf_score_shard_lse.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), vp, ctypes.c_size_t, vp]
     dll.spf_score_shard_apply.restype = i32
@@ -294,6 +304,62 @@ def spf_score_paged(prompts: Sequence[PagedPromptBuffers], workspace: torch.Tens
     _check(lib.spf_score_paged(ctypes.byref(shape), arr, len(prompts), workspace.data_ptr(),
                                workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
            "spf_score_paged")
+
+
+@dataclasses.dataclass
+class Fp8PromptBuffers:
+    """Device buffers of one prompt whose key cache is held in 8 bits (see spf_fp8_prompt in include/spf.h)."""
+    q: torch.Tensor                      # bf16 [L, Hq, m, d]
+    k_layers: Sequence[torch.Tensor]     # L tensors uint8 [Hkv, N, d] (E4M3 bytes); last dim contiguous
+    k_scale: torch.Tensor                # fp32 [L, Hkv]
+    importance: torch.Tensor             # fp32 [N] (out)
+    lse: Optional[torch.Tensor] = None   # fp32 [L, Hq, m] (out)
+
+
+def _marshal_fp8(prompts: Sequence[Fp8PromptBuffers], softmax_scale: float):
+    L, Hq, m, d = prompts[0].q.shape
+    Hkv = prompts[0].k_layers[0].shape[0]
+    shape = _Shape(L, Hq, Hkv, d, m, float(softmax_scale))
+    arr = (_Fp8Prompt * len(prompts))()
+    keep = []
+    for i, p in enumerate(prompts):
+        _dev(p.q, torch.bfloat16, "q")
+        _dev(p.k_scale, torch.float32, "k_scale")
+        _dev(p.importance, torch.float32, "importance")
+        k0 = p.k_layers[0]
+        n = k0.shape[1]
+        if len(p.k_layers) != L or not p.q.is_contiguous() or tuple(p.q.shape) != (L, Hq, m, d):
+            raise ValueError("one key tensor per layer and a contiguous q of the batch's shape")
+        for kl in p.k_layers:
+            _dev(kl, torch.uint8, "k_layers[l]")
+            if tuple(kl.shape) != (Hkv, n, d) or kl.stride(2) != 1 or kl.stride() != k0.stride():
+                raise ValueError("every k_layers[l] must be uint8 [Hkv, N, d] with a contiguous last dim and equal strides")
+        if p.k_scale.numel() != L * Hkv or not p.k_scale.is_contiguous() or p.importance.numel() != n:
+            raise ValueError("k_scale must be contiguous fp32 [L, Hkv] and importance fp32 [N]")
+        if p.lse is not None:
+            _dev(p.lse, torch.float32, "lse")
+        ptrs = (ctypes.c_void_p * L)(*[kl.data_ptr() for kl in p.k_layers])
+        keep.append(ptrs)
+        arr[i] = _Fp8Prompt(n, ctypes.cast(ptrs, ctypes.POINTER(ctypes.c_void_p)), k0.stride(0), k0.stride(1),
+                            p.k_scale.data_ptr(), p.q.data_ptr(), p.importance.data_ptr(), _ptr(p.lse))
+    return shape, arr, keep
+
+
+def spf_score_fp8_workspace_bytes(prompts: Sequence[Fp8PromptBuffers], softmax_scale: float = 0.0) -> int:
+    shape, arr, _keep = _marshal_fp8(prompts, softmax_scale)
+    n = int(lib.spf_score_fp8_workspace_bytes(ctypes.byref(shape), arr, len(prompts)))
+    if n == 0:
+        raise SpfError(-1, "spf_score_fp8_workspace_bytes", spf_last_error())
+    return n
+
+
+def spf_score_fp8(prompts: Sequence[Fp8PromptBuffers], workspace: torch.Tensor, softmax_scale: float = 0.0,
+                  dev_status: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_score for key caches held as E4M3 bytes with one fp32 scale per (layer, kv-head)."""
+    shape, arr, _keep = _marshal_fp8(prompts, softmax_scale)
+    _check(lib.spf_score_fp8(ctypes.byref(shape), arr, len(prompts), workspace.data_ptr(),
+                             workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
+           "spf_score_fp8")
 
 
 def spf_score_shard_lse(prompt: PromptBuffers, workspace: torch.Tensor, softmax_scale: float = 0.0,
@@ -544,6 +610,20 @@ class Selector:
         if self.workspace is None or self.workspace.numel() < need:
             self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
         spf_score_paged([bufs], self.workspace, self.softmax_scale, self.dev_status, stream)
+        return self._select(n, token_ids, char_start, char_end, keep, stream)
+
+    def run_fp8(self, q: torch.Tensor, k_layers: Sequence[torch.Tensor], k_scale: torch.Tensor, token_ids: torch.Tensor,
+                char_start: torch.Tensor, char_end: torch.Tensor, keep: float,
+                stream: Optional[torch.cuda.Stream] = None) -> Selection:
+        """run() for a prompt whose key cache is held as E4M3 bytes (see Fp8PromptBuffers)."""
+        n = k_layers[0].shape[1]
+        if n > self.max_tokens:
+            raise ValueError(f"prompt has {n} tokens, selector was sized for {self.max_tokens}")
+        bufs = Fp8PromptBuffers(q, k_layers, k_scale, self.importance[:n], self.lse)
+        need = spf_score_fp8_workspace_bytes([bufs], self.softmax_scale)
+        if self.workspace is None or self.workspace.numel() < need:
+            self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        spf_score_fp8([bufs], self.workspace, self.softmax_scale, self.dev_status, stream)
         return self._select(n, token_ids, char_start, char_end, keep, stream)
 
     def _select(self, n: int, token_ids: torch.Tensor, char_start: torch.Tensor, char_end: torch.Tensor, keep: float,

@@ -14,7 +14,7 @@ thread_local char g_error[512] = "";
 std::atomic<int> g_score_path{0};  // 0 automatic, 1 general two-sweep path, 2 fused path
 
 // Builds the per-prompt problem description; returns a status and leaves the reason in the error text.
-int32_t make_problem(const spf_shape* shape, const spf_prompt& pr, int32_t index, ScoreProblem* out) {
+int32_t make_problem(const spf_shape* shape, const spf_prompt& pr, int32_t index, ScoreProblem* out, int k_align = 16) {
   ScoreProblem p{};
   p.n_layers = shape->n_layers;
   p.n_q_heads = shape->n_q_heads;
@@ -54,8 +54,8 @@ int32_t make_problem(const spf_shape* shape, const spf_prompt& pr, int32_t index
   for (int l = 0; l < p.n_layers; ++l) {
     const void* kp = pr.k_layers[l];
     if (kp == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: k_layers[%d] is null", index, l);
-    if (reinterpret_cast<uintptr_t>(kp) % 16 != 0)
-      return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: k_layers[%d] is not 16-byte aligned", index, l);
+    if (reinterpret_cast<uintptr_t>(kp) % k_align != 0)
+      return fail(SPF_ERR_INVALID_ARG, "spf_score: prompt %d: k_layers[%d] is not %d-byte aligned", index, l, k_align);
     p.k.p[l] = static_cast<const __nv_bfloat16*>(kp);
   }
   p.n_tokens = pr.n_tokens;
@@ -65,6 +65,7 @@ int32_t make_problem(const spf_shape* shape, const spf_prompt& pr, int32_t index
   p.importance = pr.importance;
   p.lse_out = pr.lse;
   p.extra_lse = nullptr;
+  p.k_scale = nullptr;
   p.block_table = nullptr;
   p.block_tokens = 0;
   p.n_pool_blocks = 0;
@@ -238,6 +239,72 @@ extern "C" int32_t spf_score_paged(const spf_shape* shape, const spf_paged_promp
     const bool fused = path == 2 || (path == 0 && score_fused_supported(p, sm_count));
     const int32_t st = fused ? score_fused_launch(p, workspace, sm_count, dev_status, stream)
                              : score_mma_launch(p, workspace, sm_count, stream);
+    if (st != SPF_OK) return st;
+  }
+  return SPF_OK;
+}
+
+// 8-bit key cache: described as a bf16 prompt over the same pointers (the checks are the same: strides count elements,
+// i.e. bytes here, rows must start 8-byte aligned), then marked with its scales.
+static int32_t make_fp8_problem(const spf_shape* shape, const spf_fp8_prompt& fp, int32_t index, ScoreProblem* out) {
+  if (fp.k_scale == nullptr) return fail(SPF_ERR_INVALID_ARG, "spf_score_fp8: prompt %d: k_scale is null", index);
+  spf_prompt flat{};
+  flat.n_tokens = fp.n_tokens;
+  flat.k_layers = fp.k_layers;
+  flat.k_stride_head = fp.k_stride_head;
+  flat.k_stride_tok = fp.k_stride_tok;
+  flat.q = fp.q;
+  flat.importance = fp.importance;
+  flat.lse = fp.lse;
+  const int32_t st = make_problem(shape, flat, index, out, 8);      // rows of 8-bit keys are read 8 bytes at a time
+  if (st != SPF_OK) return st;
+  out->k_scale = fp.k_scale;
+  return SPF_OK;
+}
+
+extern "C" size_t spf_score_fp8_workspace_bytes(const spf_shape* shape, const spf_fp8_prompt* prompts, int32_t n_prompts) {
+  clear_error();
+  if (shape == nullptr || prompts == nullptr || n_prompts < 1) {
+    fail(SPF_ERR_INVALID_ARG, "spf_score_fp8_workspace_bytes: null argument or n_prompts < 1");
+    return 0;
+  }
+  size_t need = 0;
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    if (make_fp8_problem(shape, prompts[i], i, &p) != SPF_OK) return 0;
+    need = std::max(need, score_mma_workspace_bytes(p));
+  }
+  return need;
+}
+
+extern "C" int32_t spf_score_fp8(const spf_shape* shape, const spf_fp8_prompt* prompts, int32_t n_prompts, void* workspace,
+                                 size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  clear_error();
+  (void)dev_status;   // the general kernels report no device-side condition
+  if (shape == nullptr || prompts == nullptr || n_prompts < 1)
+    return fail(SPF_ERR_INVALID_ARG, "spf_score_fp8: null argument or n_prompts < 1");
+  if (g_score_path.load(std::memory_order_relaxed) == 2)
+    return fail(SPF_ERR_UNSUPPORTED, "spf_score_fp8: the fused path does not read 8-bit key caches");
+  size_t need = 0;
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    const int32_t st = make_fp8_problem(shape, prompts[i], i, &p);
+    if (st != SPF_OK) return st;
+    need = std::max(need, score_mma_workspace_bytes(p));
+  }
+  if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
+    return fail(SPF_ERR_WORKSPACE, "spf_score_fp8: workspace is null or not 256-byte aligned");
+  if (workspace_bytes < need) return fail(SPF_ERR_WORKSPACE, "spf_score_fp8: workspace has %zu bytes, %zu needed", workspace_bytes, need);
+  int sm_count = 0;
+  {
+    const int32_t st = device_sm_count(&sm_count);
+    if (st != SPF_OK) return st;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  for (int32_t i = 0; i < n_prompts; ++i) {
+    ScoreProblem p;
+    make_fp8_problem(shape, prompts[i], i, &p);
+    const int32_t st = score_mma_launch(p, workspace, sm_count, stream);
     if (st != SPF_OK) return st;
   }
   return SPF_OK;

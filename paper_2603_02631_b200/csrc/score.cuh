@@ -15,6 +15,9 @@ struct ScoreProblem {
   const __nv_bfloat16* q;
   float* importance;
   float* lse_out;  // may be null
+  // 8-bit key cache (k_scale != null): the layer pointers hold E4M3 bytes, strides count bytes, key (l, hk, s, j) has the
+  // value k_scale[l * Hkv + hk] * E4M3(byte); only the general path reads this format
+  const float* k_scale;
   const float* extra_lse;  // may be null: fp32 [L][Hq][m], natural log of what the row's denominator holds besides the prompt keys
   // paged key cache (block_tokens > 0): k.p[l] is layer l's block pool, bf16 [n_pool_blocks][Hkv][block_tokens][d];
   // logical block b of the prompt sits in pool block block_table[b] (device memory)

@@ -1042,6 +1042,7 @@ constexpr int kSmemBudget = 227 * 1024 - 1024;   // dynamic shared memory we may
 FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
   FusedPlan pl;
   const int g = p.group;
+  if (p.k_scale != nullptr) return pl;        // 8-bit key caches: general path only
   if (!(g == 1 || g == 2 || g == 4 || g == 8)) return pl;
   if (p.n_layers > kFusedMaxLayers) return pl;
   const int rows = g * p.n_lookahead;

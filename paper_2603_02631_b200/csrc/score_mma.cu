@@ -43,6 +43,28 @@ __device__ __forceinline__ uint4 load_key16(const __nv_bfloat16* p) {
   return v;
 }
 
+// Eight E4M3 keys (8 bytes) -> eight bf16 values in the same order.  Exact: every E4M3 number, subnormals included,
+// is an fp16 number (hardware conversion), and has at most four significant bits, so fp16 -> fp32 -> bf16 rounds nothing.
+__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint16_t two) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(two));
+  const __half2 h = *reinterpret_cast<const __half2*>(&h2);
+  const float2 f = __half22float2(h);
+  const __nv_bfloat162 b = __floats2bfloat162_rn(f.x, f.y);
+  return *reinterpret_cast<const uint32_t*>(&b);
+}
+
+__device__ __forceinline__ uint4 load_key8_fp8(const uint8_t* p) {
+  uint2 raw;
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(raw.x), "=r"(raw.y) : "l"(p));
+  uint4 v;
+  v.x = e4m3x2_to_bf16x2((uint16_t)(raw.x & 0xffffu));
+  v.y = e4m3x2_to_bf16x2((uint16_t)(raw.x >> 16));
+  v.z = e4m3x2_to_bf16x2((uint16_t)(raw.y & 0xffffu));
+  v.w = e4m3x2_to_bf16x2((uint16_t)(raw.y >> 16));
+  return v;
+}
+
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint4& a, uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -73,17 +95,31 @@ __device__ __forceinline__ int64_t tile_offset(int64_t key0, int64_t stride_tok,
   return block * pv.stride_block + (key0 % pv.block_tokens) * stride_tok;
 }
 
-template <int D>
+// FP8: the cache holds E4M3 bytes (strides then count bytes); the tile is widened to bf16 as it is loaded.
+template <int D, bool FP8>
 __device__ __forceinline__ void load_key_tile(KeyTile<D>& t, const __nv_bfloat16* slab, int64_t tile_off, int64_t key0,
                                               int64_t n_tokens, int64_t stride_tok, int lane) {
 #pragma unroll
   for (int nt = 0; nt < 4; ++nt) {
     int64_t key = key0 + nt * 8 + (lane >> 2);
     key = key < n_tokens ? key : n_tokens - 1;  // ragged tail: read a valid row (of the same tile), mask later
-    const __nv_bfloat16* row = slab + tile_off + (key - key0) * stride_tok + (lane & 3) * 8;
+    if constexpr (FP8) {
+      const uint8_t* row = reinterpret_cast<const uint8_t*>(slab) + tile_off + (key - key0) * stride_tok + (lane & 3) * 8;
 #pragma unroll
-    for (int j = 0; j < D / 32; ++j) t.r[nt][j] = load_key16(row + j * 32);
+      for (int j = 0; j < D / 32; ++j) t.r[nt][j] = load_key8_fp8(row + j * 32);
+    } else {
+      const __nv_bfloat16* row = slab + tile_off + (key - key0) * stride_tok + (lane & 3) * 8;
+#pragma unroll
+      for (int j = 0; j < D / 32; ++j) t.r[nt][j] = load_key16(row + j * 32);
+    }
   }
+}
+
+// Base of the (layer, kv-head) slab: strides count elements, i.e. bytes for an 8-bit cache.
+template <bool FP8>
+__device__ __forceinline__ const __nv_bfloat16* slab_base(const __nv_bfloat16* layer, int64_t head_offset) {
+  if constexpr (FP8) return reinterpret_cast<const __nv_bfloat16*>(reinterpret_cast<const uint8_t*>(layer) + head_offset);
+  return layer + head_offset;
 }
 
 inline PagedView paged_view(const ScoreProblem& p) {
@@ -148,14 +184,15 @@ __global__ void pack_q_kernel(const __nv_bfloat16* __restrict__ q, uint4* __rest
 }
 
 // Sweep 1.  grid = (n_split, n_slabs); every warp strides over the slab's 32-key tiles.
-template <int D, int MT>
+template <int D, int MT, bool FP8>
 __global__ void __launch_bounds__(kThreads) score_lse_kernel(LayerPtrs kp, const uint4* __restrict__ qf,
                                                               float2* __restrict__ partial, int64_t n_tokens,
                                                               int64_t stride_head, int64_t stride_tok, int n_kv_heads,
-                                                              float c, PagedView pv) {
+                                                              float c, const float* __restrict__ k_scale, PagedView pv) {
   const int slab = blockIdx.y;
   const int layer = slab / n_kv_heads, hk = slab % n_kv_heads;
-  const __nv_bfloat16* kslab = kp.p[layer] + hk * stride_head;
+  const __nv_bfloat16* kslab = slab_base<FP8>(kp.p[layer], hk * stride_head);
+  if (FP8) c *= __ldg(k_scale + slab);                 // the slab's key scale multiplies every logit
   const uint4* qslab = qf + (int64_t)slab * (MT * (D / 16) * 32);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t n_tiles = (n_tokens + kTileKeys - 1) / kTileKeys;
@@ -169,11 +206,11 @@ __global__ void __launch_bounds__(kThreads) score_lse_kernel(LayerPtrs kp, const
 
   int64_t tile = (int64_t)blockIdx.x * kWarpsPerCta + warp;
   KeyTile<D> cur;
-  if (tile < n_tiles) load_key_tile<D>(cur, kslab, tile_offset(tile * kTileKeys, stride_tok, pv), tile * kTileKeys, n_tokens, stride_tok, lane);
+  if (tile < n_tiles) load_key_tile<D, FP8>(cur, kslab, tile_offset(tile * kTileKeys, stride_tok, pv), tile * kTileKeys, n_tokens, stride_tok, lane);
   while (tile < n_tiles) {
     const int64_t next = tile + stride;
     KeyTile<D> nxt;
-    if (next < n_tiles) load_key_tile<D>(nxt, kslab, tile_offset(next * kTileKeys, stride_tok, pv), next * kTileKeys, n_tokens, stride_tok, lane);
+    if (next < n_tiles) load_key_tile<D, FP8>(nxt, kslab, tile_offset(next * kTileKeys, stride_tok, pv), next * kTileKeys, n_tokens, stride_tok, lane);
 
     float acc[MT][4][4];
     tile_logits<D, MT>(acc, cur, qslab, lane);
@@ -282,12 +319,12 @@ __global__ void load_lse_kernel(const float* __restrict__ lse_in, float* __restr
 }
 
 // Sweep 2.  One warp owns 32 keys for all slabs.  NI = m_pad / 8 lookahead indices live in a thread.
-template <int D, int MT, int NI>
+template <int D, int MT, int NI, bool FP8>
 __global__ void __launch_bounds__(kThreads) score_max_kernel(LayerPtrs kp, const uint4* __restrict__ qf,
                                                               const float* __restrict__ lse2, float* __restrict__ importance,
                                                               int64_t n_tokens, int64_t stride_head, int64_t stride_tok,
                                                               int n_layers, int n_kv_heads, int group, int n_lookahead,
-                                                              float c, PagedView pv) {
+                                                              float c, const float* __restrict__ k_scale, PagedView pv) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t tile = (int64_t)blockIdx.x * kWarpsPerCta + warp;
   const int64_t n_tiles = (n_tokens + kTileKeys - 1) / kTileKeys;
@@ -303,15 +340,16 @@ __global__ void __launch_bounds__(kThreads) score_max_kernel(LayerPtrs kp, const
 
   KeyTile<D> cur;
   const int64_t tile_off = tile_offset(key0, stride_tok, pv);   // the same for every layer and kv-head
-  load_key_tile<D>(cur, kp.p[0], tile_off, key0, n_tokens, stride_tok, lane);
+  load_key_tile<D, FP8>(cur, kp.p[0], tile_off, key0, n_tokens, stride_tok, lane);
   for (int slab = 0; slab < n_slabs; ++slab) {
     KeyTile<D> nxt;
     if (slab + 1 < n_slabs) {
       const int l2 = (slab + 1) / n_kv_heads, h2 = (slab + 1) % n_kv_heads;
-      load_key_tile<D>(nxt, kp.p[l2] + h2 * stride_head, tile_off, key0, n_tokens, stride_tok, lane);
+      load_key_tile<D, FP8>(nxt, slab_base<FP8>(kp.p[l2], h2 * stride_head), tile_off, key0, n_tokens, stride_tok, lane);
     }
     float acc[MT][4][4];
     tile_logits<D, MT>(acc, cur, qf + (int64_t)slab * (MT * (D / 16) * 32), lane);
+    const float cs = FP8 ? c * __ldg(k_scale + slab) : c;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -325,7 +363,7 @@ __global__ void __launch_bounds__(kThreads) score_max_kernel(LayerPtrs kp, const
         for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
           for (int e = 0; e < 2; ++e)
-            amax[slot][nt * 2 + e] = fmaxf(amax[slot][nt * 2 + e], fmaf(acc[mt][nt][2 * b + e], c, -lse));
+            amax[slot][nt * 2 + e] = fmaxf(amax[slot][nt * 2 + e], fmaf(acc[mt][nt][2 * b + e], cs, -lse));
       }
     cur = nxt;
   }
@@ -347,16 +385,26 @@ __global__ void __launch_bounds__(kThreads) score_max_kernel(LayerPtrs kp, const
 template <int D, int MT>
 void launch_lse(const ScoreProblem& p, const uint4* qf, float2* partial, int n_split, cudaStream_t stream) {
   dim3 grid(n_split, p.n_layers * p.n_kv_heads);
-  score_lse_kernel<D, MT><<<grid, kThreads, 0, stream>>>(p.k, qf, partial, p.n_tokens, p.stride_head, p.stride_tok,
-                                                         p.n_kv_heads, p.c_log2, paged_view(p));
+  if (p.k_scale != nullptr)
+    score_lse_kernel<D, MT, true><<<grid, kThreads, 0, stream>>>(p.k, qf, partial, p.n_tokens, p.stride_head, p.stride_tok,
+                                                                 p.n_kv_heads, p.c_log2, p.k_scale, paged_view(p));
+  else
+    score_lse_kernel<D, MT, false><<<grid, kThreads, 0, stream>>>(p.k, qf, partial, p.n_tokens, p.stride_head, p.stride_tok,
+                                                                  p.n_kv_heads, p.c_log2, nullptr, paged_view(p));
 }
 
 template <int D, int MT, int NI>
 void launch_max(const ScoreProblem& p, const uint4* qf, const float* lse2, cudaStream_t stream) {
   const int64_t n_tiles = ceil_div(p.n_tokens, kTileKeys);
-  score_max_kernel<D, MT, NI><<<(unsigned)ceil_div(n_tiles, kWarpsPerCta), kThreads, 0, stream>>>(
-      p.k, qf, lse2, p.importance, p.n_tokens, p.stride_head, p.stride_tok, p.n_layers, p.n_kv_heads, p.group,
-      p.n_lookahead, p.c_log2, paged_view(p));
+  const unsigned grid = (unsigned)ceil_div(n_tiles, kWarpsPerCta);
+  if (p.k_scale != nullptr)
+    score_max_kernel<D, MT, NI, true><<<grid, kThreads, 0, stream>>>(p.k, qf, lse2, p.importance, p.n_tokens, p.stride_head,
+                                                                       p.stride_tok, p.n_layers, p.n_kv_heads, p.group,
+                                                                       p.n_lookahead, p.c_log2, p.k_scale, paged_view(p));
+  else
+    score_max_kernel<D, MT, NI, false><<<grid, kThreads, 0, stream>>>(p.k, qf, lse2, p.importance, p.n_tokens, p.stride_head,
+                                                                        p.stride_tok, p.n_layers, p.n_kv_heads, p.group,
+                                                                        p.n_lookahead, p.c_log2, nullptr, paged_view(p));
 }
 
 template <int D, int MT>

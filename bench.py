@@ -282,11 +282,50 @@ def time_score_launches(spf, sel, prompts, launches, stream):
     return a.elapsed_time(b) / launches
 
 
+def fp8_workload(spf, dev, peak, stream, name="long128k"):
+    """The long-context workload with its key cache in 8 bits (spf_score_fp8, general two-sweep kernels): the
+    algorithmic bytes are the E4M3 cache read once, the scales, Q, importance and lse."""
+    import torch
+    from workloads import CONFIGS, make_prompt, quantize_keys_e4m3
+    cfg = CONFIGS[name]
+    try:
+        prompt = make_prompt(cfg, 0, dev)
+        k8, scales = quantize_keys_e4m3(prompt.k)
+        q = prompt.q
+        n = prompt.n_tokens
+        del prompt
+        torch.cuda.empty_cache()
+        sel = spf.Selector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, n, chunk=cfg.chunk,
+                           pool_kernel=cfg.pool_kernel, device=dev)
+        bufs = spf.Fp8PromptBuffers(q, k8, scales, sel.importance[:n], sel.lse)
+        ws = torch.empty(spf.spf_score_fp8_workspace_bytes([bufs]), dtype=torch.uint8, device=dev)
+        previous = spf.spf_set_score_path(0)
+        try:
+            for _ in range(3):
+                spf.spf_score_fp8([bufs], ws)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(20):
+                spf.spf_score_fp8([bufs], ws)
+            b.record(stream)
+            torch.cuda.synchronize()
+        finally:
+            spf.spf_set_score_path(previous)
+        ms = a.elapsed_time(b) / 20
+        rows = cfg.n_layers * cfg.n_q_heads * cfg.n_lookahead
+        nbytes = cfg.k_bytes() // 2 + 4 * cfg.n_layers * cfg.n_kv_heads + rows * cfg.head_dim * 2 + 4 * n + 4 * rows
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        return {"workload": name + "_fp8", "kernels": "general two-sweep path (reads the cache twice)", "ms_per_launch": ms,
+                "achieved": gbs, "frac": gbs / peak, "algorithmic_bytes": nbytes, "tokens": n}
+    except Exception as err:
+        return {"workload": name + "_fp8", "error": str(err)[:200]}
+
+
 def secondary_workloads(spf, dev, peak, stream, names=("small32k", "wide64k", "ragged8")):
     """Scoring fraction of the HBM rate on the other workload configurations (20 launches each after 3 warm-ups)."""
     import torch
     from workloads import CONFIGS, make_prompt
-    out = []
+    out = [fp8_workload(spf, dev, peak, stream)]
     for name in names:
         cfg = CONFIGS[name]
         try:
@@ -344,13 +383,23 @@ def run_ours(args):
             if want == 2:
                 raise
     spf.spf_set_score_path(2 if fused else 1)
-    # kernels per prompt: fused: score_fused, chunk_pool, select_topk, compact_spans;
-    # general: pack_q, score_lse, merge_lse, score_max + the same three
-    launches_per_prompt = 4 if fused else 7
+    # kernels per step: scoring per prompt (fused: score_fused; general: pack_q, score_lse, merge_lse, score_max), then
+    # chunk_pool, select_topk, compact_spans once per prompt, or once per batch through the batched calls
+    score_launches = 1 if fused else 4
     score_kernels = "score_fused_kernel" if fused else "pack_q + score_lse + merge_lse + score_max"
+    if n_prompts > 1:
+        bsel = spf.BatchSelector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, cfg.lengths,
+                                 chunk=cfg.chunk, pool_kernel=cfg.pool_kernel, device=dev)
+        launches_per_step = score_launches * n_prompts + 3
 
-    def step():
-        for p in prompts:
+        def step():
+            bsel.run(prompts, keep)
+    else:
+        bsel = None
+        launches_per_step = score_launches + 3
+
+        def step():
+            p = prompts[0]
             sel.run(p.q, p.k, p.token_ids, p.char_start, p.char_end, keep)
 
     def barrier():
@@ -374,7 +423,7 @@ def run_ours(args):
     t_end.record(stream)
     barrier()
     ms_total = t_start.elapsed_time(t_end)
-    status = int(sel.dev_status.item())
+    status = int((bsel or sel).dev_status.item())
     if status != 0:
         raise RuntimeError(f"device status {status} ({spf.spf_status_string(status)}) after the timed region")
 
@@ -421,7 +470,7 @@ def run_ours(args):
                       ce=p.char_end.cpu().pin_memory())
             h2d += hp["q"].numel() * 2 + sum(x.numel() * 2 for x in hp["k"]) + 3 * 4 * p.n_tokens
             host.append(hp)
-        del prompts, bufs
+        del prompts, bufs, bsel
         torch.cuda.empty_cache()
 
         def e2e_step():
@@ -469,7 +518,7 @@ def run_ours(args):
                    "l2": "inputs larger than L2 (key cache streamed every step)", "parallelism": f"prompts x{world}"},
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"], "span": "timed steps + the spf_score-only launches, 10 ms period"},
-        "gpu_launches": launches_per_prompt * n_prompts * args.steps,
+        "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "kernel": f"spf_score ({score_kernels})",
                      "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                      "frac": achieved / peak, "traffic": ncu_traffic(cfg.name, "fused" if fused else "general"), "ms_per_launch": score_ms_avg,

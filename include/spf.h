@@ -311,6 +311,46 @@ SPF_API int32_t spf_compact_spans(const int32_t* kept_chunks, int64_t k, int32_t
                                   int32_t* out_char_spans, int64_t* out_counts, void* cuda_stream);
 
 /*
+ * Batched forms of the three selection calls (Algorithm 1 runs AvgPool1D ... MapDraftChunksToTextSpans per prompt; a
+ * serving step has many prompts).  `items` is a HOST array of n_items descriptors, read during the call only; every
+ * pointer inside a descriptor is DEVICE memory with the layout and size the single-prompt call states.  One launch
+ * serves up to 32 prompts (more are split into several launches); results are identical to n_items single calls.
+ * pool_kernel and chunk are shared by the batch.  Errors as the single-prompt calls, reported with the item index
+ * before anything is launched.
+ */
+typedef struct {
+  const float* importance; /* fp32 [n_tokens]                  */
+  int64_t n_tokens;
+  float* chunk_scores;     /* out: fp32 [ceil(n_tokens / chunk)] */
+} spf_pool_item;
+
+typedef struct {
+  const float* chunk_scores; /* fp32 [n_chunks] */
+  int64_t n_chunks;
+  int64_t k;
+  int32_t* kept_chunks;      /* out: int32 [k], ascending */
+} spf_topk_item;
+
+typedef struct {
+  const int32_t* kept_chunks;
+  int64_t k;
+  int64_t n_tokens;
+  const int32_t* token_ids;
+  const int32_t* char_start;
+  const int32_t* char_end;
+  int32_t* out_ids;
+  int32_t* out_pos;          /* may be NULL */
+  int32_t* out_tok_spans;
+  int32_t* out_char_spans;
+  int64_t* out_counts;
+} spf_compact_item;
+
+SPF_API int32_t spf_chunk_pool_batch(const spf_pool_item* items, int32_t n_items, int32_t pool_kernel, int32_t chunk,
+                                     void* cuda_stream);
+SPF_API int32_t spf_select_topk_batch(const spf_topk_item* items, int32_t n_items, void* cuda_stream);
+SPF_API int32_t spf_compact_spans_batch(const spf_compact_item* items, int32_t n_items, int32_t chunk, void* cuda_stream);
+
+/*
  * Variants for two points the paper leaves open (Algorithm 1 names the operations, Appendix A.3 gives kernel 13 and
  * the chunk sizes, nothing else).  Same arguments, layouts and errors as the calls they extend.
  *

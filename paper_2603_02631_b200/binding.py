@@ -40,6 +40,22 @@ class _Fp8Prompt(ctypes.Structure):
                 ("q", ctypes.c_void_p), ("importance", ctypes.c_void_p), ("lse", ctypes.c_void_p)]
 
 
+class _PoolItem(ctypes.Structure):
+    _fields_ = [("importance", ctypes.c_void_p), ("n_tokens", ctypes.c_int64), ("chunk_scores", ctypes.c_void_p)]
+
+
+class _TopkItem(ctypes.Structure):
+    _fields_ = [("chunk_scores", ctypes.c_void_p), ("n_chunks", ctypes.c_int64), ("k", ctypes.c_int64),
+                ("kept_chunks", ctypes.c_void_p)]
+
+
+class _CompactItem(ctypes.Structure):
+    _fields_ = [("kept_chunks", ctypes.c_void_p), ("k", ctypes.c_int64), ("n_tokens", ctypes.c_int64),
+                ("token_ids", ctypes.c_void_p), ("char_start", ctypes.c_void_p), ("char_end", ctypes.c_void_p),
+                ("out_ids", ctypes.c_void_p), ("out_pos", ctypes.c_void_p), ("out_tok_spans", ctypes.c_void_p),
+                ("out_char_spans", ctypes.c_void_p), ("out_counts", ctypes.c_void_p)]
+
+
 class _SelectParams(ctypes.Structure):
     _fields_ = [("chunk", ctypes.c_int32), ("pool_kernel", ctypes.c_int32), ("keep_ratio", ctypes.c_double)]
 
@@ -95,6 +111,12 @@ def _load() -> ctypes.CDLL:
     dll.spf_compress_host.restype = i32
     dll.spf_compress_host.argtypes = [ctypes.POINTER(_Shape), i64, ctypes.POINTER(ctypes.c_void_p), vp, vp, vp, vp,
                                       ctypes.POINTER(_SelectParams), vp, ctypes.c_size_t, vp, vp, vp, vp, vp, vp]
+    dll.spf_chunk_pool_batch.restype = i32
+    dll.spf_chunk_pool_batch.argtypes = [ctypes.POINTER(_PoolItem), i32, i32, i32, vp]
+    dll.spf_select_topk_batch.restype = i32
+    dll.spf_select_topk_batch.argtypes = [ctypes.POINTER(_TopkItem), i32, vp]
+    dll.spf_compact_spans_batch.restype = i32
+    dll.spf_compact_spans_batch.argtypes = [ctypes.POINTER(_CompactItem), i32, i32, vp]
     dll.spf_keep_count.restype = i64
     dll.spf_keep_count.argtypes = [i64, ctypes.c_double]
     dll.spf_keep_rate.restype = ctypes.c_double
@@ -471,6 +493,59 @@ def spf_compact_spans(kept_chunks: torch.Tensor, k: int, chunk: int, n_tokens: i
                                  _stream_ptr(stream)), "spf_compact_spans")
 
 
+def spf_chunk_pool_batch(importances: Sequence[torch.Tensor], pool_kernel: int, chunk: int,
+                         chunk_scores: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_chunk_pool for several prompts in one launch: importances[p] fp32 [N_p] -> chunk_scores[p] fp32 [ceil(N_p / chunk)]."""
+    items = (_PoolItem * len(importances))()
+    for i, (imp, cs) in enumerate(zip(importances, chunk_scores)):
+        _dev(imp, torch.float32, "importance")
+        _dev(cs, torch.float32, "chunk_scores")
+        if chunk >= 1 and cs.numel() < (imp.numel() + chunk - 1) // chunk:
+            raise ValueError("chunk_scores is too small")
+        items[i] = _PoolItem(imp.data_ptr(), imp.numel(), cs.data_ptr())
+    _check(lib.spf_chunk_pool_batch(items, len(importances), pool_kernel, chunk, _stream_ptr(stream)), "spf_chunk_pool_batch")
+
+
+def spf_select_topk_batch(chunk_scores: Sequence[torch.Tensor], n_chunks: Sequence[int], ks: Sequence[int],
+                          kept_chunks: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_select_topk for several prompts in one launch (one CTA per prompt)."""
+    items = (_TopkItem * len(chunk_scores))()
+    for i, (cs, n, k, kept) in enumerate(zip(chunk_scores, n_chunks, ks, kept_chunks)):
+        _dev(cs, torch.float32, "chunk_scores")
+        _dev(kept, torch.int32, "kept_chunks")
+        if cs.numel() < n or kept.numel() < k:
+            raise ValueError("chunk_scores or kept_chunks is too small")
+        items[i] = _TopkItem(cs.data_ptr(), n, k, kept.data_ptr())
+    _check(lib.spf_select_topk_batch(items, len(chunk_scores), _stream_ptr(stream)), "spf_select_topk_batch")
+
+
+def spf_compact_spans_batch(kept_chunks: Sequence[torch.Tensor], ks: Sequence[int], chunk: int, n_tokens: Sequence[int],
+                            token_ids: Sequence[torch.Tensor], char_start: Sequence[torch.Tensor],
+                            char_end: Sequence[torch.Tensor], out_ids: Sequence[torch.Tensor],
+                            out_pos: Sequence[Optional[torch.Tensor]], out_tok_spans: Sequence[torch.Tensor],
+                            out_char_spans: Sequence[torch.Tensor], out_counts: Sequence[torch.Tensor],
+                            stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_compact_spans for several prompts in one launch; buffer sizes per prompt as for the single call."""
+    n_items = len(kept_chunks)
+    items = (_CompactItem * n_items)()
+    for i in range(n_items):
+        k, n = ks[i], n_tokens[i]
+        for name, t in (("kept_chunks", kept_chunks[i]), ("token_ids", token_ids[i]), ("char_start", char_start[i]),
+                        ("char_end", char_end[i]), ("out_ids", out_ids[i]), ("out_tok_spans", out_tok_spans[i]),
+                        ("out_char_spans", out_char_spans[i])):
+            _dev(t, torch.int32, name)
+        _dev(out_counts[i], torch.int64, "out_counts")
+        need = min(max(k, 0) * max(chunk, 0), n)
+        if out_ids[i].numel() < need or (out_pos[i] is not None and out_pos[i].numel() < need) or \
+                out_tok_spans[i].numel() < 2 * k or out_char_spans[i].numel() < 2 * k or out_counts[i].numel() < 2 or \
+                min(token_ids[i].numel(), char_start[i].numel(), char_end[i].numel()) < n or kept_chunks[i].numel() < k:
+            raise ValueError("a buffer is smaller than include/spf.h requires")
+        items[i] = _CompactItem(kept_chunks[i].data_ptr(), k, n, token_ids[i].data_ptr(), char_start[i].data_ptr(),
+                                char_end[i].data_ptr(), out_ids[i].data_ptr(), _ptr(out_pos[i]), out_tok_spans[i].data_ptr(),
+                                out_char_spans[i].data_ptr(), out_counts[i].data_ptr())
+    _check(lib.spf_compact_spans_batch(items, n_items, chunk, _stream_ptr(stream)), "spf_compact_spans_batch")
+
+
 def _host(t: torch.Tensor, dtype: torch.dtype, name: str) -> torch.Tensor:
     if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
         raise TypeError(f"{name} must be a contiguous host tensor of dtype {dtype}")
@@ -708,3 +783,44 @@ class Selector:
         n_kept, n_spans = int(counts[0]), int(counts[1])
         return dict(ids=ids[:n_kept].numpy().copy(), pos=pos[:n_kept].numpy().copy(), tok_spans=tok[:n_spans].numpy().copy(),
                     char_spans=ch[:n_spans].numpy().copy())
+
+
+class BatchSelector:
+    """The path for a batch of prompts of one geometry: one spf_score call for the batch, then ONE launch each of
+    pooling, top-k and compaction for all prompts (the batched calls).  Buffers are allocated once per prompt slot."""
+
+    def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, n_lookahead: int,
+                 max_tokens: Sequence[int], chunk: int = 32, pool_kernel: int = 13, softmax_scale: float = 0.0,
+                 device: str = "cuda"):
+        self.geom = (n_layers, n_q_heads, n_kv_heads, head_dim, n_lookahead)
+        self.chunk, self.pool_kernel, self.softmax_scale = chunk, pool_kernel, softmax_scale
+        self.device = torch.device(device)
+        self.slots = [Selector(n_layers, n_q_heads, n_kv_heads, head_dim, n_lookahead, n, chunk=chunk,
+                               pool_kernel=pool_kernel, softmax_scale=softmax_scale, device=device) for n in max_tokens]
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self.workspace: Optional[torch.Tensor] = None
+
+    def run(self, prompts, keep: float, stream: Optional[torch.cuda.Stream] = None):
+        """prompts: objects with q, k (list), token_ids, char_start, char_end, n_tokens (device tensors).  Returns one
+        Selection per prompt; nothing is synchronised."""
+        if len(prompts) > len(self.slots):
+            raise ValueError("more prompts than slots")
+        slots = self.slots[:len(prompts)]
+        bufs = [PromptBuffers(p.q, p.k, s.importance[:p.n_tokens], s.lse) for p, s in zip(prompts, slots)]
+        need = spf_score_workspace_bytes(bufs, self.softmax_scale)
+        if self.workspace is None or self.workspace.numel() < need:
+            self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        spf_score(bufs, self.workspace, self.softmax_scale, self.dev_status, stream)
+        ns = [p.n_tokens for p in prompts]
+        ncs = [(n + self.chunk - 1) // self.chunk for n in ns]
+        ks = [spf_keep_count(c, keep) for c in ncs]
+        spf_chunk_pool_batch([s.importance[:n] for s, n in zip(slots, ns)], self.pool_kernel, self.chunk,
+                             [s.chunk_scores[:c] for s, c in zip(slots, ncs)], stream)
+        spf_select_topk_batch([s.chunk_scores for s in slots], ncs, ks, [s.kept for s in slots], stream)
+        spf_compact_spans_batch([s.kept for s in slots], ks, self.chunk, ns, [p.token_ids for p in prompts],
+                                [p.char_start for p in prompts], [p.char_end for p in prompts], [s.out_ids for s in slots],
+                                [s.out_pos for s in slots], [s.tok_spans for s in slots], [s.char_spans for s in slots],
+                                [s.counts for s in slots], stream)
+        L, Hq, _, _, m = self.geom
+        return [Selection(s.importance[:n], s.lse.view(L, Hq, m), s.chunk_scores[:c], k, s.kept, s.out_ids, s.out_pos,
+                          s.tok_spans, s.char_spans, s.counts) for s, n, c, k in zip(slots, ns, ncs, ks)]

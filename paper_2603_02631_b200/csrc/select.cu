@@ -1,5 +1,7 @@
 // Chunk pooling, top-k chunk selection and span compaction (Appendix A.1.2, Section 3.2).
 // These steps touch a few hundred KB at most; they are latency-bound and each is a single launch.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace spf {
@@ -11,9 +13,9 @@ namespace {
 // ------------------------------------------------------------------------------------------------
 constexpr int kPoolWarps = 8;
 
-__global__ void __launch_bounds__(kPoolWarps * 32) chunk_pool_kernel(const float* __restrict__ importance, int64_t n_tokens,
-                                                                      int half, float inv_w, int chunk, bool in_range_divisor,
-                                                                      float* __restrict__ chunk_scores, int64_t n_chunks) {
+__device__ __forceinline__ void chunk_pool_body(const float* __restrict__ importance, int64_t n_tokens, int half, float inv_w,
+                                                int chunk, bool in_range_divisor, float* __restrict__ chunk_scores,
+                                                int64_t n_chunks) {
   const int lane = threadIdx.x & 31;
   const int64_t j = (int64_t)blockIdx.x * kPoolWarps + (threadIdx.x >> 5);
   if (j >= n_chunks) return;
@@ -30,6 +32,30 @@ __global__ void __launch_bounds__(kPoolWarps * 32) chunk_pool_kernel(const float
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
   if (lane == 0) chunk_scores[j] = sum / (float)(hi - lo);
+}
+
+__global__ void __launch_bounds__(kPoolWarps * 32) chunk_pool_kernel(const float* __restrict__ importance, int64_t n_tokens,
+                                                                      int half, float inv_w, int chunk, bool in_range_divisor,
+                                                                      float* __restrict__ chunk_scores, int64_t n_chunks) {
+  chunk_pool_body(importance, n_tokens, half, inv_w, chunk, in_range_divisor, chunk_scores, n_chunks);
+}
+
+// Batched calls: up to kBatchItems prompts per launch, their descriptors passed by value; blockIdx.y picks the prompt.
+constexpr int kBatchItems = 32;
+struct PoolBatch {
+  spf_pool_item item[kBatchItems];
+};
+struct TopkBatch {
+  spf_topk_item item[kBatchItems];
+};
+struct CompactBatch {
+  spf_compact_item item[kBatchItems];
+};
+
+__global__ void __launch_bounds__(kPoolWarps * 32) chunk_pool_batch_kernel(const __grid_constant__ PoolBatch b, int half, float inv_w,
+                                                                            int chunk) {
+  const spf_pool_item& it = b.item[blockIdx.y];
+  chunk_pool_body(it.importance, it.n_tokens, half, inv_w, chunk, false, it.chunk_scores, (it.n_tokens + chunk - 1) / chunk);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -69,8 +95,8 @@ __device__ __forceinline__ int block_exclusive_count(bool flag, int* warp_counts
   return before + within;
 }
 
-__global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* __restrict__ scores, int n, int k, int force,
-                                                                    int32_t* __restrict__ kept) {
+__device__ __forceinline__ void select_topk_body(const float* __restrict__ scores, int n, int k, int force,
+                                                 int32_t* __restrict__ kept) {
   __shared__ int hist[256];
   __shared__ int warp_counts[kTopkThreads / 32];
   __shared__ uint32_t sh_prefix;
@@ -146,6 +172,16 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
   }
 }
 
+__global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* __restrict__ scores, int n, int k, int force,
+                                                                    int32_t* __restrict__ kept) {
+  select_topk_body(scores, n, k, force, kept);
+}
+
+__global__ void __launch_bounds__(kTopkThreads) select_topk_batch_kernel(const __grid_constant__ TopkBatch b) {
+  const spf_topk_item& it = b.item[blockIdx.x];
+  select_topk_body(it.chunk_scores, (int)it.n_chunks, (int)it.k, 0, it.kept_chunks);
+}
+
 // ------------------------------------------------------------------------------------------------
 // spf_compact_spans.  Kept chunk r (ascending order) starts at output offset r * c because only the
 // very last chunk of the prompt can be short and, if kept, it is the last one kept.  Block 0 finds
@@ -154,7 +190,7 @@ __global__ void __launch_bounds__(kTopkThreads) select_topk_kernel(const float* 
 // ------------------------------------------------------------------------------------------------
 constexpr int kCompactThreads = 256;
 
-__global__ void __launch_bounds__(kCompactThreads) compact_spans_kernel(
+__device__ __forceinline__ void compact_spans_body(
     const int32_t* __restrict__ kept, int k, int chunk, int64_t n_tokens, const int32_t* __restrict__ token_ids,
     const int32_t* __restrict__ char_start, const int32_t* __restrict__ char_end, int32_t* __restrict__ out_ids,
     int32_t* __restrict__ out_pos, int32_t* __restrict__ out_tok_spans, int32_t* __restrict__ out_char_spans,
@@ -218,6 +254,22 @@ __global__ void __launch_bounds__(kCompactThreads) compact_spans_kernel(
     out_ids[o] = token_ids[s];
     if (out_pos != nullptr) out_pos[o] = (int32_t)s;
   }
+}
+
+__global__ void __launch_bounds__(kCompactThreads) compact_spans_kernel(
+    const int32_t* __restrict__ kept, int k, int chunk, int64_t n_tokens, const int32_t* __restrict__ token_ids,
+    const int32_t* __restrict__ char_start, const int32_t* __restrict__ char_end, int32_t* __restrict__ out_ids,
+    int32_t* __restrict__ out_pos, int32_t* __restrict__ out_tok_spans, int32_t* __restrict__ out_char_spans,
+    int64_t* __restrict__ out_counts) {
+  compact_spans_body(kept, k, chunk, n_tokens, token_ids, char_start, char_end, out_ids, out_pos, out_tok_spans, out_char_spans,
+                     out_counts);
+}
+
+__global__ void __launch_bounds__(kCompactThreads) compact_spans_batch_kernel(const __grid_constant__ CompactBatch b, int chunk) {
+  const spf_compact_item& it = b.item[blockIdx.y];
+  if ((int64_t)blockIdx.x > 1 + (it.k + kCompactThreads / 32 - 1) / (kCompactThreads / 32)) return;
+  compact_spans_body(it.kept_chunks, (int)it.k, chunk, it.n_tokens, it.token_ids, it.char_start, it.char_end, it.out_ids, it.out_pos,
+                     it.out_tok_spans, it.out_char_spans, it.out_counts);
 }
 
 }  // namespace
@@ -304,5 +356,83 @@ extern "C" int32_t spf_compact_spans(const int32_t* kept_chunks, int64_t k, int3
       kept_chunks, (int)k, chunk, n_tokens, token_ids, char_start, char_end, out_ids, out_pos, out_tok_spans, out_char_spans,
       out_counts);
   SPF_CUDA_CHECK(cudaGetLastError());
+  return SPF_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ batched calls
+extern "C" int32_t spf_chunk_pool_batch(const spf_pool_item* items, int32_t n_items, int32_t pool_kernel, int32_t chunk,
+                                        void* cuda_stream) {
+  clear_error();
+  if (items == nullptr || n_items < 1) return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool_batch: null items or n_items < 1");
+  if (pool_kernel < 1 || pool_kernel > 255 || pool_kernel % 2 == 0)
+    return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool_batch: pool_kernel must be odd and in [1, 255] (got %d)", pool_kernel);
+  if (chunk < 1) return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool_batch: chunk must be >= 1 (got %d)", chunk);
+  for (int32_t i = 0; i < n_items; ++i) {
+    if (items[i].importance == nullptr || items[i].chunk_scores == nullptr)
+      return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool_batch: item %d: null pointer", i);
+    if (items[i].n_tokens < 1) return fail(SPF_ERR_INVALID_ARG, "spf_chunk_pool_batch: item %d: n_tokens must be >= 1", i);
+    if (ceil_div(ceil_div(items[i].n_tokens, chunk), kPoolWarps) > 0x7fffffff)
+      return fail(SPF_ERR_UNSUPPORTED, "spf_chunk_pool_batch: item %d: too many chunks", i);
+  }
+  for (int32_t i0 = 0; i0 < n_items; i0 += kBatchItems) {
+    const int cnt = std::min<int32_t>(kBatchItems, n_items - i0);
+    PoolBatch b{};
+    int64_t blocks = 1;
+    for (int i = 0; i < cnt; ++i) {
+      b.item[i] = items[i0 + i];
+      blocks = std::max(blocks, ceil_div(ceil_div(items[i0 + i].n_tokens, chunk), kPoolWarps));
+    }
+    chunk_pool_batch_kernel<<<dim3((unsigned)blocks, (unsigned)cnt), kPoolWarps * 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        b, pool_kernel / 2, 1.0f / (float)pool_kernel, chunk);
+    SPF_CUDA_CHECK(cudaGetLastError());
+  }
+  return SPF_OK;
+}
+
+extern "C" int32_t spf_select_topk_batch(const spf_topk_item* items, int32_t n_items, void* cuda_stream) {
+  clear_error();
+  if (items == nullptr || n_items < 1) return fail(SPF_ERR_INVALID_ARG, "spf_select_topk_batch: null items or n_items < 1");
+  for (int32_t i = 0; i < n_items; ++i) {
+    if (items[i].chunk_scores == nullptr || items[i].kept_chunks == nullptr)
+      return fail(SPF_ERR_INVALID_ARG, "spf_select_topk_batch: item %d: null pointer", i);
+    if (items[i].n_chunks < 1 || items[i].n_chunks > 0x7fffffff || items[i].k < 1 || items[i].k > items[i].n_chunks)
+      return fail(SPF_ERR_INVALID_ARG, "spf_select_topk_batch: item %d: need 1 <= k <= n_chunks < 2^31 (k=%lld, n_chunks=%lld)", i,
+                  (long long)items[i].k, (long long)items[i].n_chunks);
+  }
+  for (int32_t i0 = 0; i0 < n_items; i0 += kBatchItems) {
+    const int cnt = std::min<int32_t>(kBatchItems, n_items - i0);
+    TopkBatch b{};
+    for (int i = 0; i < cnt; ++i) b.item[i] = items[i0 + i];
+    select_topk_batch_kernel<<<cnt, kTopkThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(b);
+    SPF_CUDA_CHECK(cudaGetLastError());
+  }
+  return SPF_OK;
+}
+
+extern "C" int32_t spf_compact_spans_batch(const spf_compact_item* items, int32_t n_items, int32_t chunk, void* cuda_stream) {
+  clear_error();
+  if (items == nullptr || n_items < 1) return fail(SPF_ERR_INVALID_ARG, "spf_compact_spans_batch: null items or n_items < 1");
+  if (chunk < 1) return fail(SPF_ERR_INVALID_ARG, "spf_compact_spans_batch: chunk must be >= 1 (got %d)", chunk);
+  for (int32_t i = 0; i < n_items; ++i) {
+    const spf_compact_item& it = items[i];
+    if (it.kept_chunks == nullptr || it.token_ids == nullptr || it.char_start == nullptr || it.char_end == nullptr ||
+        it.out_ids == nullptr || it.out_tok_spans == nullptr || it.out_char_spans == nullptr || it.out_counts == nullptr)
+      return fail(SPF_ERR_INVALID_ARG, "spf_compact_spans_batch: item %d: null pointer", i);
+    if (it.n_tokens < 1 || it.n_tokens > 0x7fffffff)
+      return fail(SPF_ERR_INVALID_ARG, "spf_compact_spans_batch: item %d: n_tokens must be in [1, 2^31)", i);
+    if (it.k < 1 || it.k > ceil_div(it.n_tokens, chunk))
+      return fail(SPF_ERR_INVALID_ARG, "spf_compact_spans_batch: item %d: k must be in [1, n_chunks]", i);
+  }
+  for (int32_t i0 = 0; i0 < n_items; i0 += kBatchItems) {
+    const int cnt = std::min<int32_t>(kBatchItems, n_items - i0);
+    CompactBatch b{};
+    int64_t blocks = 2;
+    for (int i = 0; i < cnt; ++i) {
+      b.item[i] = items[i0 + i];
+      blocks = std::max(blocks, 1 + ceil_div(items[i0 + i].k, kCompactThreads / 32));
+    }
+    compact_spans_batch_kernel<<<dim3((unsigned)blocks, (unsigned)cnt), kCompactThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(b, chunk);
+    SPF_CUDA_CHECK(cudaGetLastError());
+  }
   return SPF_OK;
 }

@@ -66,6 +66,10 @@ def parse_args():
                     help="length of the back-to-back spf_score loop behind the `sustained` record (0: skip)")
     ap.add_argument("--no-secondary", action="store_true", help="skip the scoring fractions of the other workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--parallelism", default="prompts", choices=["prompts", "keys"],
+                    help="prompts: every rank scores its own prompts (no collective); keys: ONE prompt's keys are split over "
+                         "the ranks in chunk-aligned ranges and the ranks exchange row log-sum-exps, pooling halos, chunk "
+                         "scores and selections")
     ap.add_argument("--score-path", default="auto", choices=["auto", "general", "fused"],
                     help="kernels behind spf_score: fused single-kernel path, general two-sweep path, or automatic")
     return ap.parse_args()
@@ -544,10 +548,101 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------------------------- one prompt over N ranks
+def run_keys(args, ops=None, device=None, backend="nccl", cfg=None):
+    """One prompt whose keys are split over the ranks (paper_2603_02631_b200.sharded): a step is sharded_select on every
+    rank, i.e. shard log-sum-exps -> all-reduce -> shard importance -> halo / chunk-score / selection all-gathers.  The
+    total work is fixed as the ranks grow ("strong" scaling).  `ops`, `device`, `backend` and `cfg` exist so that the same
+    code can be driven on CPU ranks (gloo) with a stand-in for the kernels; the defaults are the CUDA library over NCCL."""
+    import torch
+    import torch.distributed as dist
+    from paper_2603_02631_b200.sharded import LibraryOps, Shard, shard_bounds, sharded_select
+    from workloads import CONFIGS, make_prompt
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    on_gpu = device is None
+    if on_gpu:
+        torch.cuda.set_device(local_rank)
+        device = f"cuda:{local_rank}"
+    own_group = not dist.is_initialized()
+    if own_group:
+        if on_gpu:
+            dist.init_process_group(backend, rank=rank, world_size=world, device_id=torch.device(device))
+        else:
+            dist.init_process_group(backend, rank=rank, world_size=world)
+    cfg = cfg or CONFIGS[args.workload]
+    if len(cfg.lengths) != 1:
+        raise SystemExit("--parallelism keys splits ONE prompt: pick a single-prompt workload")
+    keep = cfg.keep[0]
+    prompt = make_prompt(cfg, 0, device)                    # the same seeded bytes on every rank; each keeps its range
+    n = prompt.n_tokens
+    lo, hi = shard_bounds(n, world, cfg.chunk)[rank]
+    shard = Shard(lo, hi, prompt.q, [k[:, lo:hi].contiguous() for k in prompt.k], prompt.token_ids[lo:hi].contiguous(),
+                  prompt.char_start[lo:hi].contiguous(), prompt.char_end[lo:hi].contiguous())
+    del prompt
+    if on_gpu:
+        torch.cuda.empty_cache()
+    if ops is None:
+        import paper_2603_02631_b200 as spf
+        ops = LibraryOps()
+        k_count = spf.spf_keep_count((n + cfg.chunk - 1) // cfg.chunk, keep)
+    else:
+        import math
+        n_chunks = (n + cfg.chunk - 1) // cfg.chunk
+        k_count = max(1, min(n_chunks, math.ceil(keep * n_chunks - 1e-9)))
+
+    def step():
+        return sharded_select(shard, n, k_count, ops, chunk=cfg.chunk, pool_kernel=cfg.pool_kernel)
+
+    def barrier():
+        dist.barrier()
+        if on_gpu:
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3) if on_gpu else args.warmup):
+        step()
+    barrier()
+    if on_gpu:
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+    t0 = time.perf_counter()
+    last = None
+    for _ in range(args.steps):
+        last = step()
+    if on_gpu:
+        b.record()
+    barrier()
+    ms_total = a.elapsed_time(b) if on_gpu else (time.perf_counter() - t0) * 1e3
+    (ms_total,) = max_over_ranks([ms_total], device, world)
+    line = None
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": n * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "bf16 in, f32 accumulate/softmax", "data": "synthetic",
+            "config": {"workload": cfg.name, "n_tokens": [n], "n_layers": cfg.n_layers, "n_q_heads": cfg.n_q_heads,
+                       "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim, "n_lookahead": cfg.n_lookahead, "chunk": cfg.chunk,
+                       "keep": keep, "pool_kernel": cfg.pool_kernel, "parallelism": f"keys x{world}",
+                       "keys_per_rank": [hi_ - lo_ for lo_, hi_ in shard_bounds(n, world, cfg.chunk)],
+                       "exchange": "max + sum all-reduce of L*Hq*m floats, all-gathers of pooling halos, chunk scores, selections",
+                       "kernels": "general two-sweep kernels, one sweep per phase" if on_gpu else "stand-in"},
+            "kept_chunks": int(last.kept.numel()), "kept_tokens": int(last.ids.numel()), "spans": int(last.tok_spans.shape[0]),
+            "gpu_launches": (9 * args.steps) if on_gpu else 0,
+        }
+        print(json.dumps(line), flush=True)
+    if own_group:
+        dist.destroy_process_group()
+    return line
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.parallelism == "keys":
+        run_keys(args)
     else:
         run_ours(args)
 

@@ -228,6 +228,19 @@ SPF_API int32_t spf_score_shard_apply(const spf_shape* shape, const spf_prompt* 
                                       size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The same two calls on the kernels spf_score would pick (spf_set_score_path applies): where the shard's shape allows it,
+ * the fused kernel runs with one of its two visits only -- spf_score_shard_lse_ex streams the shard's keys once and
+ * leaves the row log-sum-exps, spf_score_shard_apply_ex streams them once and leaves the importance -- so a rank reads
+ * its keys at the fused kernel's rate instead of the general kernels'.  `dev_status` as for spf_score: a row sum of the
+ * first call can overflow fp32 (SPF_ERR_RANGE: repeat that call with spf_score_shard_lse), a bounded wait can run out
+ * (SPF_ERR_TIMEOUT).  Workspace: spf_score_workspace_bytes for the shard.
+ */
+SPF_API int32_t spf_score_shard_lse_ex(const spf_shape* shape, const spf_prompt* prompt, void* workspace, size_t workspace_bytes,
+                                       int32_t* dev_status, void* cuda_stream);
+SPF_API int32_t spf_score_shard_apply_ex(const spf_shape* shape, const spf_prompt* prompt, const float* lse, void* workspace,
+                                         size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
  * Chooses the kernels behind spf_score, process-wide: 0 = automatic (the fused single-kernel path when
  * the shape allows it, else the general two-sweep path), 1 = always the general path, 2 = always the
  * fused path (spf_score then returns SPF_ERR_UNSUPPORTED for shapes outside it: G not in {1,2,4,8},

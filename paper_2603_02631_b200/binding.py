@@ -90,6 +90,10 @@ def _load() -> ctypes.CDLL:
     dll.spf_score_shard_lse.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), vp, ctypes.c_size_t, vp]
     dll.spf_score_shard_apply.restype = i32
     dll.spf_score_shard_apply.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), vp, vp, ctypes.c_size_t, vp]
+    dll.spf_score_shard_lse_ex.restype = i32
+    dll.spf_score_shard_lse_ex.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), vp, ctypes.c_size_t, vp, vp]
+    dll.spf_score_shard_apply_ex.restype = i32
+    dll.spf_score_shard_apply_ex.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Prompt), vp, vp, ctypes.c_size_t, vp, vp]
     dll.spf_selftest_bounded_wait.restype = i32
     dll.spf_selftest_bounded_wait.argtypes = [vp, vp]
     dll.spf_set_score_path.restype = i32
@@ -404,6 +408,30 @@ def spf_score_shard_apply(prompt: PromptBuffers, lse_all: torch.Tensor, workspac
         raise ValueError("lse_all must be contiguous fp32 [L, Hq, m]")
     _check(lib.spf_score_shard_apply(ctypes.byref(shape), arr, lse_all.data_ptr(), workspace.data_ptr(),
                                      workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "spf_score_shard_apply")
+
+
+def spf_score_shard_lse_ex(prompt: PromptBuffers, workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                           softmax_scale: float = 0.0, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_score_shard_lse on the kernels spf_score would pick (the fused kernel's first visit where the shape allows)."""
+    if prompt.lse is None:
+        raise ValueError("prompt.lse receives the result")
+    shape, arr, _keep = _marshal([prompt], softmax_scale)
+    _check(lib.spf_score_shard_lse_ex(ctypes.byref(shape), arr, workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                      _ptr(dev_status), _stream_ptr(stream)), "spf_score_shard_lse_ex")
+
+
+def spf_score_shard_apply_ex(prompt: PromptBuffers, lse_all: torch.Tensor, workspace: torch.Tensor,
+                             dev_status: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                             stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_score_shard_apply on the kernels spf_score would pick (the fused kernel's second visit where the shape allows)."""
+    _dev(lse_all, torch.float32, "lse_all")
+    shape, arr, _keep = _marshal([prompt], softmax_scale)
+    L, Hq, m, _ = prompt.q.shape
+    if lse_all.numel() != L * Hq * m or not lse_all.is_contiguous():
+        raise ValueError("lse_all must be contiguous fp32 [L, Hq, m]")
+    _check(lib.spf_score_shard_apply_ex(ctypes.byref(shape), arr, lse_all.data_ptr(), workspace.data_ptr(),
+                                        workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream_ptr(stream)),
+           "spf_score_shard_apply_ex")
 
 
 def spf_selftest_bounded_wait(dev_status: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:

@@ -312,7 +312,8 @@ extern "C" int32_t spf_score_fp8(const spf_shape* shape, const spf_fp8_prompt* p
 
 // Key-sharded scoring: the two sweeps of the general path as separate calls.
 static int32_t score_shard(const spf_shape* shape, const spf_prompt* prompt, int phase, const float* lse_in, void* workspace,
-                           size_t workspace_bytes, void* cuda_stream, const char* who) {
+                           size_t workspace_bytes, void* cuda_stream, const char* who, bool allow_fused = false,
+                           int32_t* dev_status = nullptr) {
   clear_error();
   if (shape == nullptr || prompt == nullptr) return fail(SPF_ERR_INVALID_ARG, "%s: null argument", who);
   spf_prompt pr = *prompt;
@@ -328,13 +329,16 @@ static int32_t score_shard(const spf_shape* shape, const spf_prompt* prompt, int
   if (st != SPF_OK) return st;
   if (phase == 1) p.importance = nullptr;
   if (phase == 2) p.lse_out = nullptr;
-  const size_t need = score_mma_workspace_bytes(p);
+  const size_t need = std::max(score_mma_workspace_bytes(p), score_fused_workspace_bytes(p));
   if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
     return fail(SPF_ERR_WORKSPACE, "%s: workspace is null or not 256-byte aligned", who);
   if (workspace_bytes < need) return fail(SPF_ERR_WORKSPACE, "%s: workspace has %zu bytes, %zu needed", who, workspace_bytes, need);
   int sm_count = 0;
   const int32_t sc = device_sm_count(&sm_count);
   if (sc != SPF_OK) return sc;
+  const int path = g_score_path.load(std::memory_order_relaxed);
+  if (allow_fused && (path == 2 || (path == 0 && score_fused_supported(p, sm_count))))
+    return score_fused_launch(p, workspace, sm_count, dev_status, static_cast<cudaStream_t>(cuda_stream), phase, lse_in);
   return score_mma_launch_phase(p, workspace, sm_count, phase, lse_in, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -346,6 +350,16 @@ extern "C" int32_t spf_score_shard_lse(const spf_shape* shape, const spf_prompt*
 extern "C" int32_t spf_score_shard_apply(const spf_shape* shape, const spf_prompt* prompt, const float* lse, void* workspace,
                                          size_t workspace_bytes, void* cuda_stream) {
   return score_shard(shape, prompt, 2, lse, workspace, workspace_bytes, cuda_stream, "spf_score_shard_apply");
+}
+
+extern "C" int32_t spf_score_shard_lse_ex(const spf_shape* shape, const spf_prompt* prompt, void* workspace, size_t workspace_bytes,
+                                          int32_t* dev_status, void* cuda_stream) {
+  return score_shard(shape, prompt, 1, nullptr, workspace, workspace_bytes, cuda_stream, "spf_score_shard_lse_ex", true, dev_status);
+}
+
+extern "C" int32_t spf_score_shard_apply_ex(const spf_shape* shape, const spf_prompt* prompt, const float* lse, void* workspace,
+                                            size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  return score_shard(shape, prompt, 2, lse, workspace, workspace_bytes, cuda_stream, "spf_score_shard_apply_ex", true, dev_status);
 }
 
 extern "C" int32_t spf_selftest_bounded_wait(int32_t* dev_status, void* cuda_stream) {

@@ -42,7 +42,10 @@ constexpr int kFusedMaxLayers = 64;
 constexpr int kFusedMaxCtas = 256;  // upper bound on the persistent grid
 bool score_fused_supported(const ScoreProblem& p, int sm_count);
 size_t score_fused_workspace_bytes(const ScoreProblem& p);
-int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count, int32_t* dev_status, cudaStream_t stream);
+// mode 0: the whole computation; 1: first visit only: row log-sum-exps over the given keys to p.lse_out (p.importance unused);
+// 2: second visit only, with the rows' log-sum-exps `lse_in` (device, natural log, [L][Hq][m]) supplied by the caller
+int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count, int32_t* dev_status, cudaStream_t stream, int mode = 0,
+                           const float* lse_in = nullptr);
 
 // spf_score with the kernel path given for this call only (0 automatic, 1 general, 2 fused) instead of the process-wide setting.
 int32_t score_on_path(const spf_shape* shape, const spf_prompt* prompts, int32_t n_prompts, void* workspace, size_t workspace_bytes,

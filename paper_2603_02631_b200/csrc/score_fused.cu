@@ -80,6 +80,8 @@ struct FusedArgs {
   const __nv_bfloat16* q;
   int64_t n_tokens, stride_head, stride_tok;
   int n_layers, n_kv_heads, n_lookahead, n_tiles, tiles_per_cta_max, lag, k_stages, t_stages;
+  int mode;               // 0: the whole computation; 1: first visit only (row log-sum-exps of these keys); 2: second visit only
+  const float* lse_in;    // mode 2: row log-sum-exps supplied by the caller, natural log, [L][Hq][m]
   float c, inv_c;
   unsigned long long* limbs;  // [slab][NCOLS][kLimbStride] exact fixed-point sums of exp2(c*q.k - ref) over all keys
   unsigned* counters;     // [slab] CTAs whose share of the slab's row sums is in the accumulators
@@ -551,7 +553,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       const uint64_t policy = v == 0 ? l2_policy_keep() : l2_policy_drop();
       bool ok = true;
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
-        const bool valid = v == 0 ? t < n_slabs : t >= a.lag;
+        const bool valid = v == 0 ? (t < n_slabs && a.mode != 2) : (t >= a.lag && a.mode != 1);
         const int slab = v == 0 ? t : t - a.lag;
         if (!(ok = mbar_wait(bars.q_empty(qr.stage), qr.phase ^ 1u, ab))) break;
         if (valid) {
@@ -593,7 +595,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       const uint64_t q_desc0 = smem_desc(smem_u32(q_tiles));
       bool ok = true;
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
-        const bool v1 = t < n_slabs, v2 = t >= a.lag;
+        const bool v1 = t < n_slabs && a.mode != 2, v2 = t >= a.lag && a.mode != 1;
         if (!(ok = mbar_wait_warp(bars.q_full(qr.stage), qr.phase, ab))) break;
         const uint64_t bd0 = q_desc0 + (uint64_t)((qr.stage * 2 * kQSlotBytes) >> 4);
         for (int lt = 0; lt < my_tiles; ++lt) {
@@ -641,6 +643,27 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     for (int slab = 0; ok && slab < n_slabs; ++slab) {
       const int x = 2 + (slab & 1);
       const int use = slab >> 1;                                // how often slot x was written before
+      if (a.mode == 2) {
+        // the row log-sum-exps come from the caller: no sums of our own to wait for
+        float value[2] = {0.f, 0.f};
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const int row = lane + 32 * r;
+          if (row < rows_real)
+            value[r] = __ldg(a.lse_in + ((int64_t)slab * G + row % G) * a.n_lookahead + row / G) * kLog2e * a.inv_c;
+        }
+        if (use > 0) {
+          if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const int row = lane + 32 * r;
+          if (row < NCOLS) rowoff[x * 64 + row] = value[r];
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars.o_ready(x));
+        continue;
+      }
       if (!(ok = __all_sync(0xffffffffu, count_wait(a.counters + slab, (unsigned)n_cta, ab)))) break;
       unsigned long long w[2][kLimbs];
 #pragma unroll
@@ -680,6 +703,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
           if (cta == 0 && a.lse_out != nullptr) a.lse_out[out_idx] = lse2 * kLn2;
         }
       }
+      if (a.mode == 1) continue;                                 // no second visit: nobody reads the offsets
       if (use > 0) {
         if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
       }
@@ -705,7 +729,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       sample_block = min(max((int64_t)__ldg(a.block_table + sample_key / a.block_tokens), (int64_t)0), a.n_pool_blocks - 1);
       sample_row = sample_key % a.block_tokens;
     }
-    for (int slab = 0; ok && slab < n_slabs + 2; ++slab) {
+    for (int slab = 0; ok && slab < n_slabs + 2 && a.mode != 2; ++slab) {
       if (slab < n_slabs) {
         const int x = slab & 1;
         const int use = slab >> 1;
@@ -785,8 +809,8 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
     bool ok = true;
     if (is_sum) {
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
-        if (t >= n_slabs) {
-          // nothing to sum any more: keep the stage hand-over going
+        if (t >= n_slabs || a.mode == 2) {
+          // nothing to sum (any more): keep the stage hand-over going
           for (int lt = 0; lt < my_tiles; ++lt) {
             if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
             if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
@@ -911,13 +935,13 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         tmem_store_wait();
       }
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
-        if (t < a.lag) {
+        if (t < a.lag || a.mode == 1) {
           for (int lt = 0; lt < my_tiles; ++lt) {
             if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
             if (lane == 0) mbar_arrive(bars.t_empty(tr.stage));
             tr.advance();
           }
-          if (ok && t < n_slabs) ok = reduce_slab(t);
+          if (ok && t < n_slabs && a.mode != 2) ok = reduce_slab(t);
           continue;
         }
         const int slab = t - a.lag, x2 = 2 + (slab & 1);
@@ -970,14 +994,14 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
         if (!ok) break;
         __syncwarp();
         if (lane == 0) mbar_arrive(bars.o_free(x2));
-        if (t < n_slabs) ok = reduce_slab(t);
+        if (t < n_slabs && a.mode != 2) ok = reduce_slab(t);
       }
     }
     // ---------------- importance: mean over lookahead of exp2(c * running max) ----------------
     tc_fence_before();
     if (ok) ok = es.sync(lane, ab);
     tc_fence_after();
-    if (ok && misc[0] == 0) {
+    if (ok && misc[0] == 0 && a.mode != 1) {
       // the four warps of a TMEM lane quadrant share its tiles; a thread reads all lookahead slots of its key
       constexpr int FC = NI < 16 ? NI : 16;
       const float inv_m = 1.f / (float)a.n_lookahead;
@@ -1176,7 +1200,8 @@ bool score_fused_supported(const ScoreProblem& p, int sm_count) { return make_pl
 
 size_t score_fused_workspace_bytes(const ScoreProblem& p) { return fused_workspace(p).total; }
 
-int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count, int32_t* dev_status, cudaStream_t stream) {
+int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count, int32_t* dev_status, cudaStream_t stream, int mode,
+                           const float* lse_in) {
   const FusedPlan pl = make_plan(p, sm_count);
   if (!pl.ok) return fail(SPF_ERR_UNSUPPORTED, "spf_score: shape not covered by the fused path");
   EncodeTiledFn encode = encode_fn();
@@ -1235,6 +1260,8 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   args.n_tiles = pl.n_tiles;
   args.tiles_per_cta_max = pl.tiles_per_cta_max;
   args.lag = fused_lag(p, n_slabs);
+  args.mode = mode;
+  args.lse_in = lse_in;
   args.k_stages = pl.k_stages;
   args.t_stages = pl.t_stages;
   args.c = p.c_log2;

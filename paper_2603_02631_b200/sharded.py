@@ -71,6 +71,13 @@ class LibraryOps(ShardOps):
         self.b = binding
         self.scale = softmax_scale
         self.ws: Optional[torch.Tensor] = None
+        self.status: Optional[torch.Tensor] = None
+
+    def _status(self, device) -> torch.Tensor:
+        if self.status is None:
+            self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.status.zero_()
+        return self.status
 
     def _bufs(self, shard: Shard, importance, lse):
         bufs = self.b.PromptBuffers(shard.q, shard.k_layers, importance, lse)
@@ -84,13 +91,21 @@ class LibraryOps(ShardOps):
         n = shard.hi - shard.lo
         lse = torch.empty(L * Hq * m, dtype=torch.float32, device=shard.q.device)
         scratch = torch.empty(n, dtype=torch.float32, device=shard.q.device)
-        self.b.spf_score_shard_lse(self._bufs(shard, scratch, lse), self.ws, self.scale)
+        bufs = self._bufs(shard, scratch, lse)
+        st = self._status(shard.q.device)
+        self.b.spf_score_shard_lse_ex(bufs, self.ws, st, self.scale)
+        if int(st.item()) != 0:                              # a row sum beyond fp32 or a wait that ran out: the general kernels
+            self.b.spf_score_shard_lse(bufs, self.ws, self.scale)
         return lse.view(L, Hq, m)
 
     def shard_importance(self, shard, lse_all):
         n = shard.hi - shard.lo
         imp = torch.empty(n, dtype=torch.float32, device=shard.q.device)
-        self.b.spf_score_shard_apply(self._bufs(shard, imp, None), lse_all.contiguous(), self.ws, self.scale)
+        bufs = self._bufs(shard, imp, None)
+        st = self._status(shard.q.device)
+        self.b.spf_score_shard_apply_ex(bufs, lse_all.contiguous(), self.ws, st, self.scale)
+        if int(st.item()) != 0:
+            self.b.spf_score_shard_apply(bufs, lse_all.contiguous(), self.ws, self.scale)
         return imp
 
     def smooth(self, padded, pool_kernel):

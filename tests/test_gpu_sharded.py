@@ -13,9 +13,19 @@ from workloads import bf16_bits, make_prompt, small_config
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["general", "fused"])
+def kernel_path(request):
+    """The shard calls on the general two-sweep kernels, and on the fused kernel run one visit at a time."""
+    import paper_2603_02631_b200 as mod
+    previous = mod.spf_set_score_path({"general": 1, "fused": 2}[request.param])
+    yield request.param
+    mod.spf_set_score_path(previous)
+
+
 @pytest.mark.parametrize("world", [2, 3])
-@pytest.mark.parametrize("L,Hq,Hkv,d,m,N", [(2, 8, 2, 64, 8, 5000), (2, 4, 2, 128, 16, 3333), (1, 4, 4, 64, 5, 777)])
-def test_shard_entry_points(world, L, Hq, Hkv, d, m, N):
+@pytest.mark.parametrize("L,Hq,Hkv,d,m,N", [(2, 8, 2, 64, 8, 5000), (2, 4, 2, 128, 16, 3333), (1, 4, 4, 64, 5, 777),
+                                            (3, 8, 2, 64, 16, 60001)])
+def test_shard_entry_points(kernel_path, world, L, Hq, Hkv, d, m, N):
     import paper_2603_02631_b200 as spf
     from paper_2603_02631_b200.sharded import LibraryOps, Shard, shard_bounds
     cfg = small_config("shard", n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, n_lookahead=m, lengths=(N,),

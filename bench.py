@@ -388,7 +388,7 @@ def run_ours(args):
                 raise
     spf.spf_set_score_path(2 if fused else 1)
     # kernels per step: scoring per prompt (fused: score_fused; general: pack_q, score_lse, merge_lse, score_max), then
-    # chunk_pool, select_topk, compact_spans once per prompt, or once per batch through the batched calls
+    # chunk_pool and select_compact (top-k + compaction) per prompt, or the three batched calls once per batch
     score_launches = 1 if fused else 4
     score_kernels = "score_fused_kernel" if fused else "pack_q + score_lse + merge_lse + score_max"
     if n_prompts > 1:
@@ -400,7 +400,7 @@ def run_ours(args):
             bsel.run(prompts, keep)
     else:
         bsel = None
-        launches_per_step = score_launches + 3
+        launches_per_step = score_launches + 2           # chunk_pool, then top-k and compaction in one launch
 
         def step():
             p = prompts[0]
@@ -568,6 +568,8 @@ def run_keys(args, ops=None, device=None, backend="nccl", cfg=None):
         device = f"cuda:{local_rank}"
     own_group = not dist.is_initialized()
     if own_group:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")     # a bare `python bench.py --parallelism keys` is a one-rank group
+        os.environ.setdefault("MASTER_PORT", "29577")
         if on_gpu:
             dist.init_process_group(backend, rank=rank, world_size=world, device_id=torch.device(device))
         else:
@@ -627,7 +629,7 @@ def run_keys(args, ops=None, device=None, backend="nccl", cfg=None):
                        "keep": keep, "pool_kernel": cfg.pool_kernel, "parallelism": f"keys x{world}",
                        "keys_per_rank": [hi_ - lo_ for lo_, hi_ in shard_bounds(n, world, cfg.chunk)],
                        "exchange": "max + sum all-reduce of L*Hq*m floats, all-gathers of pooling halos, chunk scores, selections",
-                       "kernels": "general two-sweep kernels, one sweep per phase" if on_gpu else "stand-in"},
+                       "kernels": "spf_score_shard_lse_ex + spf_score_shard_apply_ex (the fused kernel, one visit per call, where the shape allows)" if on_gpu else "stand-in"},
             "kept_chunks": int(last.kept.numel()), "kept_tokens": int(last.ids.numel()), "spans": int(last.tok_spans.shape[0]),
             "gpu_launches": (9 * args.steps) if on_gpu else 0,
         }

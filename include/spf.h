@@ -275,8 +275,11 @@ SPF_API int32_t spf_selftest_bounded_wait(int32_t* dev_status, void* cuda_stream
  *   - Prompts whose scratch need (spf_score_workspace_bytes gives an upper bound) exceeds
  *     SPF_STATIC_SCRATCH_BYTES are rejected with SPF_ERR_WORKSPACE before anything is launched.
  *   - The first call on each device looks up the array's device address (with that device current)
- *     and caches it.  Make that first call outside any stream capture, with the device that owns
- *     `cuda_stream` current.
+ *     and caches it.  CUDA loads a library's device code lazily, so that first lookup is also the
+ *     moment the array itself (8 MiB) comes to exist on the device: make the first call at start-up,
+ *     BEFORE the application hands the remaining HBM to its own pools (afterwards the lookup can fail
+ *     with SPF_ERR_CUDA for lack of memory), outside any stream capture, with the device that owns
+ *     `cuda_stream` current.  Any small prompt will do for that call.
  *   - Every call on a device shares the one array, and the array keeps whatever the previous call
  *     left in it.  The kernels write each scratch word before they read it, so nothing needs
  *     clearing between calls; but two calls whose kernels overlap on the GPU (different streams,
@@ -322,6 +325,17 @@ SPF_API int32_t spf_compact_spans(const int32_t* kept_chunks, int64_t k, int32_t
                                   const int32_t* token_ids, const int32_t* char_start, const int32_t* char_end,
                                   int32_t* out_ids, int32_t* out_pos, int32_t* out_tok_spans,
                                   int32_t* out_char_spans, int64_t* out_counts, void* cuda_stream);
+
+/*
+ * spf_select_topk followed by spf_compact_spans in ONE launch (Algorithm 1, TopKChunks ... MapDraftChunksToTextSpans):
+ * both steps are latency-bound, and chaining them inside one CTA saves a launch per prompt.  Arguments, layouts and
+ * results are those of the two calls (kept_chunks receives the k indices as spf_select_topk writes them); n_chunks must
+ * equal ceil(n_tokens / chunk).  Results are identical to the two separate calls.
+ */
+SPF_API int32_t spf_select_compact(const float* chunk_scores, int64_t n_chunks, int64_t k, int32_t chunk, int64_t n_tokens,
+                                   const int32_t* token_ids, const int32_t* char_start, const int32_t* char_end,
+                                   int32_t* kept_chunks, int32_t* out_ids, int32_t* out_pos, int32_t* out_tok_spans,
+                                   int32_t* out_char_spans, int64_t* out_counts, void* cuda_stream);
 
 /*
  * Batched forms of the three selection calls (Algorithm 1 runs AvgPool1D ... MapDraftChunksToTextSpans per prompt; a

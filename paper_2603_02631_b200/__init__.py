@@ -11,7 +11,7 @@ import importlib
 _BINDING_NAMES = (
     "LIB_PATH", "SpfError", "Selection", "Selector", "PromptBuffers", "PagedPromptBuffers", "spf_score_paged", "spf_score_paged_workspace_bytes", "lib", "spf_chunk_pool", "spf_chunk_pool_edge", "spf_select_topk_forced", "spf_compact_spans",
     "spf_keep_count", "spf_keep_rate", "spf_snap_budget", "spf_concat_with_delim", "spf_last_error", "spf_score", "spf_score_extra", "spf_score_shard_lse", "spf_score_shard_apply", "spf_selftest_bounded_wait", "spf_set_score_path", "spf_score_static", "spf_score_workspace_bytes", "spf_select_topk",
-    "spf_status_string", "spf_version", "spf_compress_host", "spf_compress_host_arena_bytes", "Fp8PromptBuffers", "spf_score_shard_lse_ex", "spf_score_shard_apply_ex", "BatchSelector", "spf_chunk_pool_batch", "spf_select_topk_batch", "spf_compact_spans_batch", "spf_score_fp8", "spf_score_fp8_workspace_bytes",
+    "spf_status_string", "spf_version", "spf_compress_host", "spf_compress_host_arena_bytes", "Fp8PromptBuffers", "spf_select_compact", "spf_score_shard_lse_ex", "spf_score_shard_apply_ex", "BatchSelector", "spf_chunk_pool_batch", "spf_select_topk_batch", "spf_compact_spans_batch", "spf_score_fp8", "spf_score_fp8_workspace_bytes",
 )
 __all__ = list(_BINDING_NAMES) + ["binding"]
 

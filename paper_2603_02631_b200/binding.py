@@ -115,6 +115,8 @@ def _load() -> ctypes.CDLL:
     dll.spf_compress_host.restype = i32
     dll.spf_compress_host.argtypes = [ctypes.POINTER(_Shape), i64, ctypes.POINTER(ctypes.c_void_p), vp, vp, vp, vp,
                                       ctypes.POINTER(_SelectParams), vp, ctypes.c_size_t, vp, vp, vp, vp, vp, vp]
+    dll.spf_select_compact.restype = i32
+    dll.spf_select_compact.argtypes = [vp, i64, i64, i32, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     dll.spf_chunk_pool_batch.restype = i32
     dll.spf_chunk_pool_batch.argtypes = [ctypes.POINTER(_PoolItem), i32, i32, i32, vp]
     dll.spf_select_topk_batch.restype = i32
@@ -521,6 +523,31 @@ def spf_compact_spans(kept_chunks: torch.Tensor, k: int, chunk: int, n_tokens: i
                                  _stream_ptr(stream)), "spf_compact_spans")
 
 
+def spf_select_compact(chunk_scores: torch.Tensor, n_chunks: int, k: int, chunk: int, n_tokens: int, token_ids: torch.Tensor,
+                       char_start: torch.Tensor, char_end: torch.Tensor, kept_chunks: torch.Tensor, out_ids: torch.Tensor,
+                       out_pos: Optional[torch.Tensor], out_tok_spans: torch.Tensor, out_char_spans: torch.Tensor,
+                       out_counts: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spf_select_topk + spf_compact_spans in one launch (same buffers and sizes as the two calls)."""
+    _dev(chunk_scores, torch.float32, "chunk_scores")
+    for name, t in (("kept_chunks", kept_chunks), ("token_ids", token_ids), ("char_start", char_start),
+                    ("char_end", char_end), ("out_ids", out_ids), ("out_tok_spans", out_tok_spans),
+                    ("out_char_spans", out_char_spans)):
+        _dev(t, torch.int32, name)
+    if out_pos is not None:
+        _dev(out_pos, torch.int32, "out_pos")
+    _dev(out_counts, torch.int64, "out_counts")
+    need = min(max(k, 0) * max(chunk, 0), n_tokens)
+    if chunk_scores.numel() < n_chunks or kept_chunks.numel() < k or out_ids.numel() < need or \
+            (out_pos is not None and out_pos.numel() < need) or out_tok_spans.numel() < 2 * k or \
+            out_char_spans.numel() < 2 * k or out_counts.numel() < 2 or \
+            min(token_ids.numel(), char_start.numel(), char_end.numel()) < n_tokens:
+        raise ValueError("a buffer is smaller than include/spf.h requires")
+    _check(lib.spf_select_compact(chunk_scores.data_ptr(), n_chunks, k, chunk, n_tokens, token_ids.data_ptr(),
+                                  char_start.data_ptr(), char_end.data_ptr(), kept_chunks.data_ptr(), out_ids.data_ptr(),
+                                  _ptr(out_pos), out_tok_spans.data_ptr(), out_char_spans.data_ptr(), out_counts.data_ptr(),
+                                  _stream_ptr(stream)), "spf_select_compact")
+
+
 def spf_chunk_pool_batch(importances: Sequence[torch.Tensor], pool_kernel: int, chunk: int,
                          chunk_scores: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
     """spf_chunk_pool for several prompts in one launch: importances[p] fp32 [N_p] -> chunk_scores[p] fp32 [ceil(N_p / chunk)]."""
@@ -742,10 +769,12 @@ class Selector:
         if self.force_first or self.force_last:
             k = max(k, len({0} if self.force_first else set()) + (1 if self.force_last and (n_chunks > 1 or not self.force_first) else 0))
             spf_select_topk_forced(self.chunk_scores, n_chunks, k, self.force_first, self.force_last, self.kept, stream)
+            spf_compact_spans(self.kept, k, self.chunk, n, token_ids, char_start, char_end, self.out_ids, self.out_pos,
+                              self.tok_spans, self.char_spans, self.counts, stream)
         else:
-            spf_select_topk(self.chunk_scores, n_chunks, k, self.kept, stream)
-        spf_compact_spans(self.kept, k, self.chunk, n, token_ids, char_start, char_end, self.out_ids, self.out_pos,
-                          self.tok_spans, self.char_spans, self.counts, stream)
+            # top-k and compaction chained in one launch
+            spf_select_compact(self.chunk_scores, n_chunks, k, self.chunk, n, token_ids, char_start, char_end, self.kept,
+                               self.out_ids, self.out_pos, self.tok_spans, self.char_spans, self.counts, stream)
         L, Hq, _, _, m = self.geom
         return Selection(self.importance[:n], self.lse.view(L, Hq, m), self.chunk_scores[:n_chunks], k, self.kept,
                          self.out_ids, self.out_pos, self.tok_spans, self.char_spans, self.counts)

@@ -77,7 +77,8 @@ __device__ __forceinline__ uint32_t chunk_key(const float* __restrict__ scores, 
   return order_key(scores[j]);
 }
 
-// Exclusive prefix count of `flag` over the CTA (thread order); *total gets the CTA-wide count.
+// Exclusive prefix count of `flag` over the CTA (thread order); *total gets the CTA-wide count.  The 32 warp totals
+// are scanned by warp 0 with shuffles (slot 32 of warp_counts receives the CTA-wide total).
 __device__ __forceinline__ int block_exclusive_count(bool flag, int* warp_counts, int* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned ballot = __ballot_sync(0xffffffffu, flag);
@@ -85,23 +86,48 @@ __device__ __forceinline__ int block_exclusive_count(bool flag, int* warp_counts
   __syncthreads();  // warp_counts may still be read from the previous use
   if (lane == 0) warp_counts[warp] = __popc(ballot);
   __syncthreads();
-  int before = 0, all = 0;
-  for (int w = 0; w < kTopkThreads / 32; ++w) {
-    const int cnt = warp_counts[w];
-    before += w < warp ? cnt : 0;
-    all += cnt;
+  if (warp == 0) {
+    const int own = warp_counts[lane];
+    int incl = own;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += v;
+    }
+    warp_counts[lane] = incl - own;                      // exclusive offset of warp `lane`
+    if (lane == 31) warp_counts[32] = incl;
   }
-  *total = all;
-  return before + within;
+  __syncthreads();
+  *total = warp_counts[32];
+  return warp_counts[warp] + within;
+}
+
+// One histogram increment per distinct bin of a warp instead of one per thread: scores share their top bits, so the
+// first passes would otherwise send thousands of atomics to a handful of shared-memory words.
+__device__ __forceinline__ void hist_add_aggregated(int* hist, bool take, uint32_t bin) {
+  const unsigned peers = __match_any_sync(0xffffffffu, take ? bin : 0xffffffffu);
+  if (take && (int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&hist[bin], __popc(peers));
 }
 
 __device__ __forceinline__ void select_topk_body(const float* __restrict__ scores, int n, int k, int force,
                                                  int32_t* __restrict__ kept) {
   __shared__ int hist[256];
-  __shared__ int warp_counts[kTopkThreads / 32];
+  __shared__ int warp_counts[kTopkThreads / 32 + 1];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_remaining;
 
+  // up to kTopkCache keys per thread stay in registers for all passes (n <= 8192 chunks, i.e. prompts of up to 262 144
+  // tokens at chunk 32); longer score arrays are re-read from global memory in every pass
+  constexpr int kTopkCache = 8;
+  const bool cached = n <= kTopkThreads * kTopkCache;
+  uint32_t ck[kTopkCache];
+  if (cached) {
+#pragma unroll
+    for (int i = 0; i < kTopkCache; ++i) {
+      const int j = threadIdx.x + i * kTopkThreads;
+      ck[i] = j < n ? chunk_key(scores, j, n, force) : 0u;
+    }
+  }
   uint32_t prefix = 0;     // the bits of the k-th largest key found so far
   uint32_t mask = 0;       // which bits of `prefix` are fixed
   int remaining = k;       // rank of the wanted key among the keys that match the prefix
@@ -109,9 +135,19 @@ __device__ __forceinline__ void select_topk_body(const float* __restrict__ score
     const int shift = 24 - 8 * pass;
     for (int b = threadIdx.x; b < 256; b += kTopkThreads) hist[b] = 0;
     __syncthreads();
-    for (int j = threadIdx.x; j < n; j += kTopkThreads) {
-      const uint32_t key = chunk_key(scores, j, n, force);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+    if (cached) {
+#pragma unroll
+      for (int i = 0; i < kTopkCache; ++i) {
+        const int j = threadIdx.x + i * kTopkThreads;
+        if (i * kTopkThreads < n)                            // warp-uniform: whole warps take part or none
+          hist_add_aggregated(hist, j < n && (ck[i] & mask) == prefix, (ck[i] >> shift) & 255u);
+      }
+    } else {
+      for (int j0 = 0; j0 < n; j0 += kTopkThreads) {
+        const int j = j0 + threadIdx.x;
+        const uint32_t key = j < n ? chunk_key(scores, j, n, force) : 0u;
+        hist_add_aggregated(hist, j < n && (key & mask) == prefix, (key >> shift) & 255u);
+      }
     }
     __syncthreads();
     if (threadIdx.x < 32) {
@@ -157,9 +193,16 @@ __device__ __forceinline__ void select_topk_body(const float* __restrict__ score
   }
   // `prefix` is now the k-th largest key; `remaining` of the entries equal to it are kept (lowest indices).
   int out_base = 0, eq_base = 0;
-  for (int j0 = 0; j0 < n; j0 += kTopkThreads) {
+  for (int j0 = 0, it = 0; j0 < n; j0 += kTopkThreads, ++it) {
     const int j = j0 + threadIdx.x;
-    const uint32_t key = j < n ? chunk_key(scores, j, n, force) : 0u;
+    uint32_t key = 0u;
+    if (cached) {
+#pragma unroll
+      for (int i = 0; i < kTopkCache; ++i)
+        if (i == it) key = ck[i];                            // constant indices keep the cache in registers
+    } else if (j < n) {
+      key = chunk_key(scores, j, n, force);
+    }
     const bool gt = j < n && key > prefix;
     const bool eq = j < n && key == prefix;
     int eq_total, sel_total;
@@ -263,6 +306,75 @@ __global__ void __launch_bounds__(kCompactThreads) compact_spans_kernel(
     int64_t* __restrict__ out_counts) {
   compact_spans_body(kept, k, chunk, n_tokens, token_ids, char_start, char_end, out_ids, out_pos, out_tok_spans, out_char_spans,
                      out_counts);
+}
+
+// ------------------------------------------------------------------------------------------------
+// spf_select_compact: top-k and compaction of one prompt in ONE CTA (the two steps are latency-bound and the second
+// only needs the first's k indices, so a second launch costs more than the work).  After the selection the same
+// 1024 threads find the runs of consecutive kept chunks (a prefix count of run starts, as compact_spans_kernel's
+// block 0 does) and copy ids and positions, one warp per kept chunk.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kTopkThreads) select_compact_kernel(
+    const float* __restrict__ scores, int n, int k, int chunk, int64_t n_tokens, const int32_t* __restrict__ token_ids,
+    const int32_t* __restrict__ char_start, const int32_t* __restrict__ char_end, int32_t* __restrict__ kept,
+    int32_t* __restrict__ out_ids, int32_t* __restrict__ out_pos, int32_t* __restrict__ out_tok_spans,
+    int32_t* __restrict__ out_char_spans, int64_t* __restrict__ out_counts) {
+  select_topk_body(scores, n, k, 0, kept);
+  __threadfence_block();
+  __syncthreads();                                          // kept[0..k) is complete and visible to the whole CTA
+  __shared__ int warp_counts[kTopkThreads / 32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int32_t* kv = kept;                                 // written by other threads of this CTA a moment ago: read past L1
+  int span_base = 0;
+  for (int r0 = 0; r0 < k; r0 += kTopkThreads) {
+    const int r = r0 + threadIdx.x;
+    int64_t j = -1;
+    bool starts = false, ends = false;
+    if (r < k) {
+      j = __ldcg(kv + r);
+      starts = r == 0 || __ldcg(kv + r - 1) + 1 != j;
+      ends = r == k - 1 || __ldcg(kv + r + 1) != j + 1;
+    }
+    const unsigned ballot = __ballot_sync(0xffffffffu, starts);
+    const int within = __popc(ballot & ((2u << lane) - 1u));  // inclusive
+    __syncthreads();
+    if (lane == 0) warp_counts[warp] = __popc(ballot);
+    __syncthreads();
+    int before = 0, all = 0;
+    for (int w = 0; w < kTopkThreads / 32; ++w) {
+      before += w < warp ? warp_counts[w] : 0;
+      all += warp_counts[w];
+    }
+    const int span = span_base + before + within - 1;      // index of the run this chunk belongs to
+    if (r < k) {
+      if (starts) {
+        const int64_t a = j * chunk;
+        out_tok_spans[2 * span] = (int32_t)a;
+        out_char_spans[2 * span] = char_start[a];
+      }
+      if (ends) {
+        const int64_t b = min((j + 1) * chunk, n_tokens);
+        out_tok_spans[2 * span + 1] = (int32_t)b;
+        out_char_spans[2 * span + 1] = char_end[b - 1];
+      }
+    }
+    span_base += all;
+  }
+  const int64_t last = __ldcg(kv + k - 1);
+  const int64_t n_kept = (int64_t)(k - 1) * chunk + (min((last + 1) * chunk, n_tokens) - last * chunk);
+  if (threadIdx.x == 0) {
+    out_counts[0] = n_kept;
+    out_counts[1] = span_base;
+  }
+  // kept chunk r (ascending) starts at output offset r * chunk: only the prompt's last chunk can be short.  The
+  // output is walked as one flat array so that every thread has several independent loads in flight
+#pragma unroll 4
+  for (int64_t o = threadIdx.x; o < n_kept; o += kTopkThreads) {
+    const int64_t r = o / chunk;
+    const int64_t t = (int64_t)__ldcg(kv + r) * chunk + (o - r * chunk);
+    out_ids[o] = __ldg(token_ids + t);
+    if (out_pos != nullptr) out_pos[o] = (int32_t)t;
+  }
 }
 
 __global__ void __launch_bounds__(kCompactThreads) compact_spans_batch_kernel(const __grid_constant__ CompactBatch b, int chunk) {
@@ -434,5 +546,29 @@ extern "C" int32_t spf_compact_spans_batch(const spf_compact_item* items, int32_
     compact_spans_batch_kernel<<<dim3((unsigned)blocks, (unsigned)cnt), kCompactThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(b, chunk);
     SPF_CUDA_CHECK(cudaGetLastError());
   }
+  return SPF_OK;
+}
+
+extern "C" int32_t spf_select_compact(const float* chunk_scores, int64_t n_chunks, int64_t k, int32_t chunk, int64_t n_tokens,
+                                      const int32_t* token_ids, const int32_t* char_start, const int32_t* char_end,
+                                      int32_t* kept_chunks, int32_t* out_ids, int32_t* out_pos, int32_t* out_tok_spans,
+                                      int32_t* out_char_spans, int64_t* out_counts, void* cuda_stream) {
+  clear_error();
+  if (chunk_scores == nullptr || kept_chunks == nullptr || token_ids == nullptr || char_start == nullptr || char_end == nullptr ||
+      out_ids == nullptr || out_tok_spans == nullptr || out_char_spans == nullptr || out_counts == nullptr)
+    return fail(SPF_ERR_INVALID_ARG, "spf_select_compact: null pointer");
+  if (chunk < 1) return fail(SPF_ERR_INVALID_ARG, "spf_select_compact: chunk must be >= 1 (got %d)", chunk);
+  if (n_tokens < 1 || n_tokens > 0x7fffffff)
+    return fail(SPF_ERR_INVALID_ARG, "spf_select_compact: n_tokens must be in [1, 2^31) (got %lld)", (long long)n_tokens);
+  if (n_chunks != ceil_div(n_tokens, chunk))
+    return fail(SPF_ERR_INVALID_ARG, "spf_select_compact: n_chunks must be ceil(n_tokens / chunk) (got %lld for %lld tokens)",
+                (long long)n_chunks, (long long)n_tokens);
+  if (k < 1 || k > n_chunks)
+    return fail(SPF_ERR_INVALID_ARG, "spf_select_compact: k must be in [1, n_chunks] (got k=%lld, n_chunks=%lld)", (long long)k,
+                (long long)n_chunks);
+  select_compact_kernel<<<1, kTopkThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      chunk_scores, (int)n_chunks, (int)k, chunk, n_tokens, token_ids, char_start, char_end, kept_chunks, out_ids, out_pos,
+      out_tok_spans, out_char_spans, out_counts);
+  SPF_CUDA_CHECK(cudaGetLastError());
   return SPF_OK;
 }

@@ -81,3 +81,38 @@ def test_batched_calls_validate_every_item_before_launching():
     assert err.value.status == -1 and "item 1" in str(err.value)
     with pytest.raises(spf.SpfError):
         spf.spf_chunk_pool_batch([good], 12, 32, [out])   # even pooling kernel
+
+
+@pytest.mark.parametrize("n,chunk,keep", [(10007, 32, 0.3), (131072, 32, 0.1), (262144, 32, 0.5), (5000, 128, 0.03), (31, 32, 1.0),
+                                          (300000, 32, 0.25)])
+def test_select_compact_equals_the_two_calls(n, chunk, keep):
+    """Top-k and compaction chained in one launch: bit-identical to spf_select_topk + spf_compact_spans (with ties, with the
+    score array cached in registers and, for the longest prompt, re-read per pass), and to the oracle's selection."""
+    import paper_2603_02631_b200 as spf
+    g = torch.Generator().manual_seed(n)
+    imp = torch.rand(n, generator=g)
+    imp[::7] = 0.25
+    imp = imp.cuda()
+    n_chunks = (n + chunk - 1) // chunk
+    k = spf.spf_keep_count(n_chunks, keep)
+    scores = torch.zeros(n_chunks, device="cuda")
+    spf.spf_chunk_pool(imp, 13, chunk, scores)
+    scores[::3] = scores[min(1, n_chunks - 1)].item()      # heavy ties across chunk scores
+    ids = torch.randint(0, 32000, (n,), generator=g, dtype=torch.int32).cuda()
+    starts = torch.arange(n, dtype=torch.int32, device="cuda") * 2
+    ends = starts + 1
+
+    def outs():
+        rows = min(k * chunk, n)
+        return [torch.full((k,), -1, dtype=torch.int32, device="cuda"), torch.full((rows,), -1, dtype=torch.int32, device="cuda"),
+                torch.full((rows,), -1, dtype=torch.int32, device="cuda"), torch.full((k, 2), -1, dtype=torch.int32, device="cuda"),
+                torch.full((k, 2), -1, dtype=torch.int32, device="cuda"), torch.zeros(2, dtype=torch.int64, device="cuda")]
+    a, b = outs(), outs()
+    spf.spf_select_topk(scores, n_chunks, k, a[0])
+    spf.spf_compact_spans(a[0], k, chunk, n, ids, starts, ends, a[1], a[2], a[3], a[4], a[5])
+    spf.spf_select_compact(scores, n_chunks, k, chunk, n, ids, starts, ends, b[0], b[1], b[2], b[3], b[4], b[5])
+    torch.cuda.synchronize()
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    want = oracle.select_topk(scores.cpu().numpy().astype(np.float64), k)
+    assert b[0].cpu().tolist() == want.tolist()

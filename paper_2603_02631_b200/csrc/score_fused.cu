@@ -19,11 +19,15 @@
 // and sees all query rows of it: the max over heads is in-thread.
 //
 // Warps.  0: TMA producer of the first-visit tiles.  1: MMA issuer.  2: log-sum-exp warp (turns a slab's complete
-// row sums into the offsets of visit 2).  3: reference + publisher warp.  4..11: "sum" warps, the visit-1 half of
-// every stage (exp2-bound).  12..19: "max" warps, the visit-2 half (ALU / shared-memory bound); they also add up the
-// per-key sums of the sum warps, which reach them through a shared-memory buffer once per slab.  20: TMA producer of
-// the second-visit tiles.  The two epilogue groups run independently, so the exp2 work and the max work overlap on
-// every scheduler.
+// row sums into the offsets of visit 2).  3: reference warp (hands the per-slab reference of visit 1 to the sum warps,
+// two slabs ahead).  4..11: "sum" warps, the visit-1 half of every stage (exp2-bound).  12..19: "max" warps, the
+// visit-2 half (ALU / shared-memory bound); they also add up the per-key sums of the sum warps, which reach them
+// through a shared-memory buffer once per slab.  20: TMA producer of the second-visit tiles.  21: publisher (reports
+// this CTA's finished share of a slab to the other CTAs).  The two epilogue groups run independently, so the exp2
+// work and the max work overlap on every scheduler.  The per-slab loops of warps 2, 3 and 21 are chains of memory
+// round trips; with short slabs (few tiles per CTA) such a chain, not the tiles, sets the pace as soon as it grows.
+// Hence a warp for each, and hence the references are computed once for all CTAs (each CTA a share of the slabs, at
+// the start) instead of by every CTA for every slab.
 //
 // Reference.  Visit 1 subtracts one reference per slab inside the exp2 argument: the SMALLEST logit of the slab's
 // rows against one fixed sample key, plus a margin of 60 (base-2 units).  Every row's largest logit is at least
@@ -57,8 +61,12 @@ namespace spf {
 namespace {
 
 constexpr int kTileKeys = 128;
-constexpr int kThreads = 672;          // warp 0 TMA (first visit), 1 MMA issue, 2 log-sum-exp, 3 references + publisher, 4..19 epilogue, 20 TMA (second visit)
+constexpr int kThreads = 704;          // warp 0 TMA (first visit), 1 MMA issue, 2 log-sum-exp, 3 references, 4..19 epilogue, 20 TMA (second visit), 21 publisher
 constexpr int kProducer2Warp = 20;
+#ifndef SPF_FUSED_LB
+#define SPF_FUSED_LB kThreads
+#endif
+constexpr int kPublisherWarp = 21;
 constexpr int kLimbs = 7;              // 40-bit limbs of the exact row-sum accumulators (covers every finite fp32)
 constexpr int kLimbStride = 8;         // 64-bit words per row in the accumulator array
 constexpr int kQStages = 2;
@@ -85,6 +93,7 @@ struct FusedArgs {
   float c, inv_c;
   unsigned long long* limbs;  // [slab][NCOLS][kLimbStride] exact fixed-point sums of exp2(c*q.k - ref) over all keys
   unsigned* counters;     // [slab] CTAs whose share of the slab's row sums is in the accumulators
+  unsigned* refs;         // [slab] the slab's first-visit reference (float bits, lowest bit set; zero = not computed yet)
   float* lse_out;         // optional [L][Hq][m], natural log
   const float* extra_lse; // optional [L][Hq][m], natural log: what each row's denominator holds besides the prompt keys
   float* importance;      // [N]
@@ -181,6 +190,29 @@ __device__ __forceinline__ bool count_wait(const unsigned* counter, unsigned tar
 
 
 // Waits until *flag (shared memory, written by another warp of the CTA) has reached `target`.
+// Waits until a word that starts as zero has been set (by another CTA) and returns its value in `value`.
+__device__ __forceinline__ bool word_wait(const unsigned* word, unsigned& value, const Abort& ab) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
+    if (v != 0u) {
+      value = v;
+      return true;
+    }
+    if ((it & 15u) == 15u) {
+      if (*ab.flag) return false;
+      const unsigned long long now = global_timer();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > ab.timeout_ns) {
+        record_timeout(ab);
+        return false;
+      }
+      __nanosleep(100);
+    }
+  }
+}
+
 __device__ __forceinline__ bool flag_wait(const volatile int* flag, int target, const Abort& ab) {
   unsigned long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
@@ -450,7 +482,7 @@ struct EpiSync {
 
 // ---------------------------------------------------------------------------------------------- kernel
 template <int D, int NCOLS, int G>
-__global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_constant__ FusedMaps maps,
+__global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __grid_constant__ FusedMaps maps,
                                                                    const __grid_constant__ FusedArgs a) {
   constexpr int EW = 16;                        // epilogue warps: 8 for the first visit (sums), 8 for the second (maxima)
   constexpr int EWV = EW / 2;                   // per visit: two warps per TMEM lane quadrant, half of the columns each
@@ -716,12 +748,14 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       if (lane == 0) mbar_arrive(bars.o_ready(x));
     }
   } else if (warp == 3) {
-    // ===== reference / publisher warp.  Per slab: the reference of the first visit (the smallest logit of the slab's
-    // rows against one fixed sample key, plus a margin), written as soon as the slot of slab - 2 is free; then, once
-    // the shares of slab - 2 have been added to the accumulators, orders those additions before the arrival count
-    // and reports this CTA (keeps the fence off the epilogue warps) =====
+    // ===== reference warp.  The reference of a slab's first visit is the smallest logit of the slab's rows against one
+    // fixed sample key, plus a margin.  It depends on the inputs only and is the same for every CTA, so the CTAs share
+    // the work: CTA c computes the references of slabs c, c + n_cta, ... once, at the start, and stores them in global
+    // memory (a zero word = not there yet, so a stored value has its lowest bit set: every reader sees the same
+    // number, which is all that matters for a reference).  Afterwards the warp only feeds the epilogue: 32 slabs'
+    // references are fetched at a time, one per lane, and written to the slot of slab - 2 as soon as that is free =====
     bool ok = true;
-    const int64_t sample_key = a.n_tokens / 2;                  // the same key for every CTA: one reference per slab
+    const int64_t sample_key = a.n_tokens / 2;                  // the same key for every slab and CTA
     // where that key sits: its row inside its pool block when the cache is paged (a bad table entry is clamped: this is a
     // plain load, not a bounds-checked TMA copy)
     int64_t sample_block = 0, sample_row = sample_key;
@@ -729,71 +763,92 @@ __global__ void __launch_bounds__(kThreads, 1) score_fused_kernel(const __grid_c
       sample_block = min(max((int64_t)__ldg(a.block_table + sample_key / a.block_tokens), (int64_t)0), a.n_pool_blocks - 1);
       sample_row = sample_key % a.block_tokens;
     }
-    for (int slab = 0; ok && slab < n_slabs + 2 && a.mode != 2; ++slab) {
-      if (slab < n_slabs) {
-        const int x = slab & 1;
-        const int use = slab >> 1;
-        const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
-        const uint4* krow = reinterpret_cast<const uint4*>(a.k_layers[layer] + sample_block * a.stride_block + hk * a.stride_head +
-                                                           sample_row * a.stride_tok);
-        const uint4* qrow[2];
+    constexpr int LPR = D / 8;                                  // lanes per row: 8 bf16 of it each
+    constexpr int RPP = 32 / LPR;                               // rows per pass of the warp
+    constexpr int PASSES = NCOLS / RPP;                         // 4..32
+    constexpr int BATCH = PASSES < 8 ? PASSES : 8;              // loads in flight per lane
+    for (int slab = cta; slab < n_slabs && a.mode != 2; slab += n_cta) {
+      const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
+      const uint4 kv = __ldg(reinterpret_cast<const uint4*>(a.k_layers[layer] + sample_block * a.stride_block + hk * a.stride_head +
+                                                            sample_row * a.stride_tok) + lane % LPR);
+      float kf[8];
+      {
+        const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv);
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          const int row = min(lane + 32 * r, rows_real - 1);
-          qrow[r] = reinterpret_cast<const uint4*>(a.q + (((int64_t)slab * G + row % G) * a.n_lookahead + row / G) * D);
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(k2[e]);
+          kf[2 * e] = f.x;
+          kf[2 * e + 1] = f.y;
         }
-        float dot[2] = {0.f, 0.f};
+      }
+      // the smallest sample logit of the slab's rows (padding rows repeat a real one).  The smallest, so that no row's
+      // sum can underflow (see the header).  A softmax scale is positive, so the smallest q.k is the smallest logit
+      float ref = INFINITY;
+#pragma unroll 1
+      for (int p0 = 0; p0 < PASSES; p0 += BATCH) {
+        uint4 qv[BATCH];
 #pragma unroll
-        for (int half = 0; half < D / 64; ++half) {
-          uint4 kv[8], qv[2][8];
+        for (int b = 0; b < BATCH; ++b) {
+          const int row = min((p0 + b) * RPP + lane / LPR, rows_real - 1);
+          qv[b] = __ldg(reinterpret_cast<const uint4*>(a.q + (((int64_t)slab * G + row % G) * a.n_lookahead + row / G) * D) + lane % LPR);
+        }
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch) {
-            kv[ch] = __ldg(krow + half * 8 + ch);
-            qv[0][ch] = __ldg(qrow[0] + half * 8 + ch);
-            qv[1][ch] = __ldg(qrow[1] + half * 8 + ch);
+        for (int b = 0; b < BATCH; ++b) {
+          const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv[b]);
+          float dot = 0.f;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 qf = __bfloat1622float2(q2[e]);
+            dot = fmaf(kf[2 * e], qf.x, fmaf(kf[2 * e + 1], qf.y, dot));
           }
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch) {
-            const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv[ch]);
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-              const __nv_bfloat162* q2 = reinterpret_cast<const __nv_bfloat162*>(&qv[r][ch]);
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float2 kf = __bfloat1622float2(k2[e]), qf = __bfloat1622float2(q2[e]);
-                dot[r] = fmaf(kf.x, qf.x, fmaf(kf.y, qf.y, dot[r]));
-              }
-            }
-          }
+          for (int off = LPR / 2; off >= 1; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+          ref = fminf(ref, dot);
         }
-        // one reference per slab: the smallest sample logit of its rows (padding rows repeat a real one), in base-2
-        // units, plus the margin.  The smallest, so that no row's sum can underflow (see the header).  A softmax scale
-        // is positive, so the smallest q.k is the smallest logit
-        float ref = fminf(dot[0], dot[1]);
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) ref = fminf(ref, __shfl_xor_sync(0xffffffffu, ref, off));
-        ref = fmaf(ref, a.c, kRefMargin);
-        if (use > 0) {
-          if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
-        }
-        if (lane == 0) {
-          rowoff[x * 64] = ref;
-          ref_slots[slab % kRefSlots] = ref;
-          __threadfence_block();
-          misc[3] = slab + 1;                                    // the log-sum-exp warp reads ref_slots after this
-          mbar_arrive(bars.o_ready(x));
-        }
-        __syncwarp();
       }
-      if (slab >= 2) {
-        const int ps = slab - 2;
-        if (!(ok = mbar_wait_warp(bars.pub_ready(ps % kPubSlots), (uint32_t)(ps / kPubSlots) & 1u, ab))) break;
-        if (lane == 0) {
-          __threadfence();
-          atomicAdd(a.counters + ps, 1u);
-        }
-        __syncwarp();
+#pragma unroll
+      for (int off = 16; off >= LPR; off >>= 1) ref = fminf(ref, __shfl_xor_sync(0xffffffffu, ref, off));
+      ref = fmaf(ref, a.c, kRefMargin);                          // base-2 units, plus the margin
+      if (lane == 0) {
+        const unsigned word = __float_as_uint(ref) | 1u;
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.refs + slab), "r"(word) : "memory");
       }
+    }
+    unsigned mine = 0u;                                          // lane's reference of slab (slab & ~31) + lane
+    for (int slab = 0; ok && slab < n_slabs && a.mode != 2; ++slab) {
+      if ((slab & 31) == 0) {
+        mine = 1u;
+        const bool got = slab + lane >= n_slabs || word_wait(a.refs + slab + lane, mine, ab);
+        if (!(ok = __all_sync(0xffffffffu, got))) break;
+      }
+      const float ref = __uint_as_float(__shfl_sync(0xffffffffu, mine, slab & 31));
+      const int x = slab & 1;
+      const int use = slab >> 1;
+      if (use > 0) {
+        // free since the sum warps picked up the reference of slab - 2, i.e. since they began that slab
+        if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
+      }
+      if (lane == 0) {
+        rowoff[x * 64] = ref;
+        ref_slots[slab % kRefSlots] = ref;
+        __threadfence_block();
+        misc[3] = slab + 1;                                    // the log-sum-exp warp reads ref_slots after this
+        mbar_arrive(bars.o_ready(x));
+      }
+      __syncwarp();
+    }
+  } else if (warp == kPublisherWarp) {
+    // ===== publisher warp: once this CTA's shares of a slab have been added to the accumulators, orders those
+    // additions before the arrival count and reports the CTA (keeps the fence and the atomic's round trip off the
+    // epilogue warps) =====
+    bool ok = true;
+    for (int ps = 0; ok && ps < n_slabs && a.mode != 2; ++ps) {
+      if (!(ok = mbar_wait_warp(bars.pub_ready(ps % kPubSlots), (uint32_t)(ps / kPubSlots) & 1u, ab))) break;
+      if (lane == 0) {
+        __threadfence();
+        atomicAdd(a.counters + ps, 1u);
+      }
+      __syncwarp();
     }
   } else if (warp >= 4 && warp < 4 + EW) {
     // ===== epilogue.  Warps 4..11 ("sum" warps) take the first-visit tile of every stage, warps 12..19 ("max" warps)
@@ -1104,7 +1159,7 @@ int fused_lag(const ScoreProblem& p, int n_slabs) {
 }
 
 struct FusedWorkspace {
-  size_t limbs_off, counters_off, total;   // both are cleared before every launch
+  size_t limbs_off, counters_off, refs_off, total;   // all three are cleared before every launch
 };
 
 FusedWorkspace fused_workspace(const ScoreProblem& p) {
@@ -1112,7 +1167,8 @@ FusedWorkspace fused_workspace(const ScoreProblem& p) {
   FusedWorkspace w;
   w.limbs_off = 0;
   w.counters_off = align_up(n_slabs * 64 * kLimbStride * sizeof(unsigned long long), 256);
-  w.total = align_up(w.counters_off + n_slabs * sizeof(unsigned), 256);
+  w.refs_off = align_up(w.counters_off + n_slabs * sizeof(unsigned), 256);
+  w.total = align_up(w.refs_off + n_slabs * sizeof(unsigned), 256);
   return w;
 }
 
@@ -1268,6 +1324,7 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   args.inv_c = 1.0f / p.c_log2;
   args.limbs = reinterpret_cast<unsigned long long*>(base + w.limbs_off);
   args.counters = reinterpret_cast<unsigned*>(base + w.counters_off);
+  args.refs = reinterpret_cast<unsigned*>(base + w.refs_off);
   args.lse_out = p.lse_out;
   args.extra_lse = p.extra_lse;
   args.importance = p.importance;

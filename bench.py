@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM read + write bytes of one scoring launch, from the ncu capture summarised in profiles/.  Each entry names
 # the SHA-256 of the kernel source it was taken from: once the source changes, the figure is reported as null.
 NCU_TRAFFIC = {
-    ("long128k", "fused"): {"bytes": 4 * (598066944 + 9501440), "source": "paper_2603_02631_b200/csrc/score_fused.cu",
-                            "sha256": "0c6f2db448269922e050e9062e896a09d2b311bda0ef945e47bb34e9014a1d12",
+    ("long128k", "fused"): {"bytes": 4 * (538848256 + 6746368), "source": "paper_2603_02631_b200/csrc/score_fused.cu",
+                            "sha256": "f5290961f9ccc5026dd9969a7690aeee6bf7d11599bb3aa4194f6eb22d7552f7",
                             "note": "captured on long128k_l4 (4 of 16 layers), scaled x4"},
 }
 

@@ -1150,10 +1150,12 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
 
 // How many slabs the second visit runs behind the first.  The cross-CTA hand-over of a slab's row sums takes
 // about 5 us; with short slabs (few tiles per CTA) two slabs of lead do not cover it, so the lag grows until the
-// slabs kept live for the second read (lag + 1 of them) would no longer sit comfortably in L2.
+// slabs kept live for the second read (lag + 1 of them) would no longer sit comfortably in L2: 64 MB of them, i.e.
+// three slabs of lead at 16 MB a slab (measured at 128k tokens, d = 64: lag 2..4 within 1 %, 5 and 6 cost 6 and 11 %;
+// at 64k tokens, d = 128: lag 3 best, 2 and 4 cost 9 and 3 %, 5 costs 22 %).
 int fused_lag(const ScoreProblem& p, int n_slabs) {
   const double slab_bytes = (double)p.n_tokens * p.head_dim * 2.0;
-  int lag = (int)(80.0 * 1024 * 1024 / slab_bytes) - 1;
+  int lag = (int)(64.0 * 1024 * 1024 / slab_bytes) - 1;
   lag = std::max(2, std::min(lag, 8));
   return std::max(1, std::min(lag, n_slabs));
 }

@@ -178,18 +178,25 @@ SPF_API int32_t spf_score_paged(const spf_shape* shape, const spf_paged_prompt* 
  * (l, hk, s, j) has the value
  *     k_scale[l * Hkv + hk] * E4M3(byte at k_layers[l] + hk * k_stride_head + s * k_stride_tok + j)
  * with E4M3 the 8-bit floating-point format of 1 sign, 4 exponent (bias 7) and 3 mantissa bits, subnormals, no
- * infinities (the byte patterns 0x7F / 0xFF, NaN, must not occur).  Bytes are widened to bf16 exactly and the scale is
- * folded into the softmax scale of its (layer, kv-head), so the arithmetic and its error are those of spf_score.
- * Queries stay bf16.
+ * infinities (the byte patterns 0x7F / 0xFF, NaN, must not occur).  The key scale is folded into the softmax scale of
+ * its (layer, kv-head).  Queries are given in bf16.
  *
  *   k_layers       HOST array of L device pointers (8-byte aligned), layer l uint8 [Hkv][N][d]; strides in bytes,
  *                  k_stride_tok >= d, both strides multiples of 8
  *   k_scale        DEVICE fp32 [L][Hkv], positive and finite
  *   others         as in spf_prompt
  *
- * Only the general two-sweep kernels read this format (they read the cache twice, so halving its bytes is where it
- * pays); with the fused path forced (spf_set_score_path(2)) the call returns SPF_ERR_UNSUPPORTED.  `dev_status` is
- * accepted for symmetry and never written.  Workspace: spf_score_fp8_workspace_bytes(...), rules as for spf_score.
+ * Kernel paths, chosen as in spf_score (spf_set_score_path):
+ *   fused     needs 16-byte aligned layer pointers and strides (and a shape spf_score's fused path takes).  The tensor
+ *             cores multiply the E4M3 keys by E4M3 operands only, so each bf16 query is handed to them as the sum of two
+ *             E4M3 terms after a power-of-two scaling per (layer, kv-head): exact for every element within 2^9 of the
+ *             largest |q| of its (layer, kv-head), off by at most 2^-17 of that largest value below.  Accumulation is
+ *             fp32.  Range limits and `dev_status` as for spf_score's fused path (SPF_ERR_RANGE, SPF_ERR_TIMEOUT).
+ *   general   any cache the layout rules above admit.  Bytes are widened to bf16 exactly; arithmetic and error are
+ *             those of spf_score's general path; `dev_status` is not written.
+ * With the path left automatic, caches the fused path cannot read go to the general kernels; with the fused path
+ * forced they are refused with SPF_ERR_UNSUPPORTED.  Workspace: spf_score_fp8_workspace_bytes(...), rules as for
+ * spf_score.
  */
 typedef struct {
   int64_t n_tokens;

@@ -272,7 +272,7 @@ extern "C" size_t spf_score_fp8_workspace_bytes(const spf_shape* shape, const sp
   for (int32_t i = 0; i < n_prompts; ++i) {
     ScoreProblem p;
     if (make_fp8_problem(shape, prompts[i], i, &p) != SPF_OK) return 0;
-    need = std::max(need, score_mma_workspace_bytes(p));
+    need = std::max(need, std::max(score_mma_workspace_bytes(p), score_fused_workspace_bytes(p)));
   }
   return need;
 }
@@ -280,17 +280,14 @@ extern "C" size_t spf_score_fp8_workspace_bytes(const spf_shape* shape, const sp
 extern "C" int32_t spf_score_fp8(const spf_shape* shape, const spf_fp8_prompt* prompts, int32_t n_prompts, void* workspace,
                                  size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
   clear_error();
-  (void)dev_status;   // the general kernels report no device-side condition
   if (shape == nullptr || prompts == nullptr || n_prompts < 1)
     return fail(SPF_ERR_INVALID_ARG, "spf_score_fp8: null argument or n_prompts < 1");
-  if (g_score_path.load(std::memory_order_relaxed) == 2)
-    return fail(SPF_ERR_UNSUPPORTED, "spf_score_fp8: the fused path does not read 8-bit key caches");
   size_t need = 0;
   for (int32_t i = 0; i < n_prompts; ++i) {
     ScoreProblem p;
     const int32_t st = make_fp8_problem(shape, prompts[i], i, &p);
     if (st != SPF_OK) return st;
-    need = std::max(need, score_mma_workspace_bytes(p));
+    need = std::max(need, std::max(score_mma_workspace_bytes(p), score_fused_workspace_bytes(p)));
   }
   if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0)
     return fail(SPF_ERR_WORKSPACE, "spf_score_fp8: workspace is null or not 256-byte aligned");
@@ -304,7 +301,9 @@ extern "C" int32_t spf_score_fp8(const spf_shape* shape, const spf_fp8_prompt* p
   for (int32_t i = 0; i < n_prompts; ++i) {
     ScoreProblem p;
     make_fp8_problem(shape, prompts[i], i, &p);
-    const int32_t st = score_mma_launch(p, workspace, sm_count, stream);
+    const int path = g_score_path.load(std::memory_order_relaxed);
+    const bool fused = path == 2 || (path == 0 && score_fused_supported(p, sm_count));
+    const int32_t st = fused ? score_fused_launch(p, workspace, sm_count, dev_status, stream) : score_mma_launch(p, workspace, sm_count, stream);
     if (st != SPF_OK) return st;
   }
   return SPF_OK;

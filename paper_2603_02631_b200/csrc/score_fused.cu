@@ -29,6 +29,13 @@
 // Hence a warp for each, and hence the references are computed once for all CTAs (each CTA a share of the slabs, at
 // the start) instead of by every CTA for every slab.
 //
+// 8-bit key caches (template parameter FP8): the key tiles are E4M3 bytes (rows of d bytes: 64-byte swizzle at d = 64,
+// the 128-byte one at d = 128), the instruction kind is f8f6f4 with 32 bytes of the row per instruction, and the
+// queries come as two E4M3 terms per element from split_q_kernel, accumulated into the same columns -- the same number
+// of instructions per tile as for bf16.  The factor from accumulated dot product to base-2 logit then differs per slab
+// (softmax scale x key scale / query scale), so the epilogue multiplies by a per-slab value where the bf16 kernel has
+// a constant and keeps the running maxima in base-2 logits.  The bf16 instantiations compile to what they were.
+//
 // Reference.  Visit 1 subtracts one reference per slab inside the exp2 argument: the SMALLEST logit of the slab's
 // rows against one fixed sample key, plus a margin of 60 (base-2 units).  Every row's largest logit is at least
 // its own sample logit, hence at least reference - 60, and ex2.approx.ftz only flushes terms below reference - 126,
@@ -76,10 +83,13 @@ constexpr int kRefSlots = 16;         // row references stay readable for this m
 constexpr int kPubSlots = 16;        // slabs whose hand-over to the publisher may be pending at once
 constexpr float kRefMargin = 60.f;     // base-2 units added to the sampled reference logit
 constexpr unsigned long long kTimeoutNs = 2000000000ull;
-constexpr int kSubTileBytes = kTileKeys * 128;  // 128 keys x 64 bf16, one swizzle-128B tile
+// Key rows are d bf16 (128 or 256 bytes) or d E4M3 bytes (64 or 128).  A tile is stored as sub-tiles of 128 keys x one swizzle
+// span: 128 bytes of the row (128-byte swizzle), or the whole row where it has only 64 bytes (64-byte swizzle).
+__host__ __device__ constexpr int row_bytes(int d, bool fp8) { return fp8 ? d : 2 * d; }
+__host__ __device__ constexpr int sub_row_bytes(int rowb) { return rowb > 128 ? 128 : rowb; }
 
 struct FusedMaps {
-  CUtensorMap q;                      // (d, g, i, slab) view of the query tensor
+  CUtensorMap q;                      // (d, g, i, slab) view of the query tensor; 8-bit keys: (d, row, slab * 2 + part) view of the split queries
   CUtensorMap k[kFusedMaxLayers];     // (d, key, kv-head) view of each layer's key cache
 };
 
@@ -91,6 +101,11 @@ struct FusedArgs {
   int mode;               // 0: the whole computation; 1: first visit only (row log-sum-exps of these keys); 2: second visit only
   const float* lse_in;    // mode 2: row log-sum-exps supplied by the caller, natural log, [L][Hq][m]
   float c, inv_c;
+  // 8-bit key caches: the queries reach the tensor cores as two E4M3 terms per element (see split_q_kernel), scaled per
+  // slab; slab_scale[slab] turns an accumulated dot product into base-2 logits (softmax scale, key scale and query scale
+  // in one factor) and key_scale[slab] is the key cache's own scale.  Null for bf16 caches.
+  const float* slab_scale;
+  const float* key_scale;
   unsigned long long* limbs;  // [slab][NCOLS][kLimbStride] exact fixed-point sums of exp2(c*q.k - ref) over all keys
   unsigned* counters;     // [slab] CTAs whose share of the slab's row sums is in the accumulators
   unsigned* refs;         // [slab] the slab's first-visit reference (float bits, lowest bit set; zero = not computed yet)
@@ -164,6 +179,31 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
 
 // Warp-collective form: every lane waits, and all lanes agree on the outcome (a timeout seen by one
 // lane only must not split the warp in front of .aligned instructions).
+// Waits for two barriers at once: both are polled before either answer is looked at, so that their latencies overlap.
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b, const Abort& ab) {
+  bool a = mbar_try_wait(bar_a, parity_a);
+  bool b = mbar_try_wait(bar_b, parity_b);
+  if (a && b) return true;
+  unsigned long long t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    if (!a) a = mbar_try_wait(bar_a, parity_a);
+    if (!b) b = mbar_try_wait(bar_b, parity_b);
+    if (a && b) return true;
+    if (it > 2u) __nanosleep(64);
+    if ((it & 63u) == 0u) {
+      if (*ab.flag) return false;
+      const unsigned long long now = global_timer();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > ab.timeout_ns) {
+        record_timeout(ab);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait2_warp(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b, const Abort& ab) {
+  return __all_sync(0xffffffffu, mbar_wait2(bar_a, parity_a, bar_b, parity_b, ab));
+}
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const Abort& ab) {
   return __all_sync(0xffffffffu, mbar_wait(bar, parity, ab));
 }
@@ -281,27 +321,53 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// One tensor-core instruction: M = 128 keys x N query rows x 32 bytes of the head dimension (16 bf16, or 32 E4M3 with
+// both operands in that format).
+template <bool FP8>
 __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
+  if constexpr (FP8)
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 
-// Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+// Shared-memory operand descriptor: K-major rows of SUBROW bytes (128 or 64) with the swizzle of that span, 8-row groups
+// 8 * SUBROW bytes apart.
+template <int SUBROW>
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  static_assert(SUBROW == 128 || SUBROW == 64, "swizzle span");
   uint64_t d = 0;
   d |= (uint64_t)((addr & 0x3FFFFu) >> 4);   // start address / 16
   d |= (uint64_t)1 << 16;                    // leading byte offset (not used by swizzled K-major operands)
-  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset: 8 rows x 128 bytes
+  d |= (uint64_t)((8 * SUBROW) >> 4) << 32;  // stride byte offset: 8 rows
   d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+  d |= (uint64_t)(SUBROW == 128 ? 2 : 4) << 61;   // 128-byte / 64-byte swizzle
   return d;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
-__host__ __device__ constexpr uint32_t instr_desc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileKeys >> 4) << 24);
+// One E4M3 byte as fp32 (exact).
+__device__ __forceinline__ float e4m3_to_float(uint32_t byte) {
+  uint32_t h2;
+  asm("{\n.reg .b16 lo;\ncvt.u16.u32 lo, %1;\ncvt.rn.f16x2.e4m3x2 %0, lo;\n}" : "=r"(h2) : "r"(byte & 0xffu));
+  return __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
+}
+// fp32 to the nearest E4M3 byte (saturating).
+__device__ __forceinline__ uint32_t float_to_e4m3(float x) {
+  uint32_t out;
+  asm("{\n.reg .b16 r;\ncvt.rn.satfinite.e4m3x2.f32 r, %1, %2;\ncvt.u32.u16 %0, r;\n}" : "=r"(out) : "f"(0.f), "f"(x));
+  return out & 0xffu;
+}
+
+// Instruction descriptor: bf16 x bf16 (operand format 1) or E4M3 x E4M3 (format 0) -> fp32, both operands K-major,
+// M = 128, N = n.
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool fp8) {
+  return (1u << 4) | ((fp8 ? 0u : 1u) << 7) | ((fp8 ? 0u : 1u) << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileKeys >> 4) << 24);
 }
 
 // TMEM -> registers, in two parts: tmem_issue starts the (asynchronous) load of N consecutive columns of the warp's
@@ -413,17 +479,17 @@ __device__ __forceinline__ void tmem_wait<32>(uint32_t (&r)[32]) {
 }
 
 // ---------------------------------------------------------------------------------------------- layout
-__host__ __device__ constexpr int q_sub_tile_bytes(int ncols) { return ncols * 128; }   // ncols query rows x 64 bf16
 
 struct SmemLayout {
   uint32_t k_off, q_off, xbuf_off, ref_off, rowoff_off, tileblk_off, bar_off, misc_off, total;
 };
 
-__host__ __device__ inline SmemLayout smem_layout(int d, int ncols, int group, int k_stages, int tiles_per_cta_max) {
+__host__ __device__ inline SmemLayout smem_layout(int d, bool fp8, int ncols, int group, int k_stages, int tiles_per_cta_max) {
   SmemLayout s;
   uint32_t o = 0;
-  s.k_off = o;        o += (uint32_t)k_stages * 2 * (d / 64) * kSubTileBytes;
-  s.q_off = o;        o += (uint32_t)kQStages * 2 * (d / 64) * q_sub_tile_bytes(ncols);
+  const uint32_t rowb = (uint32_t)row_bytes(d, fp8);
+  s.k_off = o;        o += (uint32_t)k_stages * 2 * kTileKeys * rowb;                 // stages of two key tiles
+  s.q_off = o;        o += (uint32_t)kQStages * 2 * (fp8 ? 2 : 1) * ncols * rowb;      // stages of two query tiles (two terms each for 8-bit keys)
   s.xbuf_off = o;     o += (uint32_t)ncols * (kTileKeys / 4) * 4;
   s.ref_off = o;      o += kRefSlots * 4;
   s.rowoff_off = o;   o += 4 * 64 * 4;
@@ -481,7 +547,7 @@ struct EpiSync {
 };
 
 // ---------------------------------------------------------------------------------------------- kernel
-template <int D, int NCOLS, int G>
+template <int D, int NCOLS, int G, bool FP8>
 __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __grid_constant__ FusedMaps maps,
                                                                    const __grid_constant__ FusedArgs a) {
   constexpr int EW = 16;                        // epilogue warps: 8 for the first visit (sums), 8 for the second (maxima)
@@ -490,11 +556,17 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
   constexpr int CHK = CW < 16 ? CW : 16;        // columns per tensor-memory load
   constexpr int NCH = CW / CHK;                 // loads per tile and thread: 1 or 2
   constexpr int NI = NCOLS / G;          // lookahead slots per key in the running-max array
-  constexpr int KSUB = D / 64;           // 64-wide sub-tiles per key tile
+  constexpr int ROWB = row_bytes(D, FP8);                   // bytes per key row: 64, 128 or 256
+  constexpr int SUBROW = sub_row_bytes(ROWB);               // the swizzle span: 128 bytes, or the whole 64-byte row
+  constexpr int KSUB = ROWB / SUBROW;                       // sub-tiles per key tile
+  constexpr int KSTEPS = SUBROW / 32;                       // tensor-core instructions per sub-tile (32 bytes of the row each)
+  constexpr int XSUB = SUBROW / (FP8 ? 1 : 2);              // elements per sub-tile row: the TMA x coordinate of sub-tile h is h * XSUB
+  constexpr int kSubTileBytes = kTileKeys * SUBROW;
   constexpr int kSlotBytes = KSUB * kSubTileBytes;          // one key tile
   constexpr int kStageBytes = 2 * kSlotBytes;               // slot 0: first-visit tile, slot 1: second-visit tile
-  constexpr int kQSub = q_sub_tile_bytes(NCOLS);
-  constexpr int kQSlotBytes = KSUB * kQSub;
+  constexpr int QPARTS = FP8 ? 2 : 1;                       // 8-bit keys: the queries come as two E4M3 terms
+  constexpr int kQSub = NCOLS * SUBROW;
+  constexpr int kQSlotBytes = QPARTS * KSUB * kQSub;
   constexpr int kTmemCols = kTmemColsAll;
   constexpr int NIH = (NCOLS / 2) / G;   // lookahead slots per max-warp thread
   constexpr int AC = NIH < 8 ? NIH : 8;  // running maxima moved per tensor-memory load / store
@@ -507,7 +579,7 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
   // 1024-byte alignment by offsetting the shared array itself, so that the compiler still knows these are
   // shared-memory addresses (a round trip through an integer would turn every access into a generic one)
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-  const SmemLayout lay = smem_layout(D, NCOLS, G, a.k_stages, a.tiles_per_cta_max);
+  const SmemLayout lay = smem_layout(D, FP8, NCOLS, G, a.k_stages, a.tiles_per_cta_max);
   unsigned char* k_tiles = smem + lay.k_off;
   unsigned char* q_tiles = smem + lay.q_off;
   float* xbuf = reinterpret_cast<float*>(smem + lay.xbuf_off);         // [NCOLS][32]: partial row sums of one slab, each over four keys
@@ -515,6 +587,7 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
   int* tile_block = reinterpret_cast<int*>(smem + lay.tileblk_off);   // paged key cache: pool block of each of the CTA's tiles
   float* rowoff = reinterpret_cast<float*>(smem + lay.rowoff_off);   // [4 slots][64]: what the epilogue subtracts per row
   volatile int* misc = reinterpret_cast<volatile int*>(smem + lay.misc_off);  // [0] abort, [1] tmem base, [3] references written
+  volatile float* slab_c = reinterpret_cast<volatile float*>(smem + lay.misc_off + 32);   // [4]: 8-bit keys: slab_scale of the slab in slot x
   const Bars bars{smem_u32(smem + lay.bar_off), a.k_stages};
   const Abort ab{misc, a.dev_status};
 
@@ -589,10 +662,18 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
         const int slab = v == 0 ? t : t - a.lag;
         if (!(ok = mbar_wait(bars.q_empty(qr.stage), qr.phase ^ 1u, ab))) break;
         if (valid) {
-          mbar_expect_tx(bars.q_full(qr.stage), (uint32_t)(KSUB * rows_real * 128));
-          for (int h = 0; h < KSUB; ++h)
-            tma_load_4d(smem_u32(q_tiles + (qr.stage * 2 + v) * kQSlotBytes + h * kQSub), &maps.q, h * 64, 0, 0, slab,
-                        bars.q_full(qr.stage));
+          if constexpr (FP8) {
+            mbar_expect_tx(bars.q_full(qr.stage), (uint32_t)kQSlotBytes);
+            for (int part = 0; part < QPARTS; ++part)
+              for (int h = 0; h < KSUB; ++h)
+                tma_load_3d(smem_u32(q_tiles + (qr.stage * 2 + v) * kQSlotBytes + (part * KSUB + h) * kQSub), &maps.q, h * XSUB, 0,
+                            slab * QPARTS + part, bars.q_full(qr.stage), policy);
+          } else {
+            mbar_expect_tx(bars.q_full(qr.stage), (uint32_t)(KSUB * rows_real * 128));
+            for (int h = 0; h < KSUB; ++h)
+              tma_load_4d(smem_u32(q_tiles + (qr.stage * 2 + v) * kQSlotBytes + h * kQSub), &maps.q, h * 64, 0, 0, slab,
+                          bars.q_full(qr.stage));
+          }
         } else {
           mbar_arrive(bars.q_full(qr.stage));
         }
@@ -606,9 +687,9 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
             for (int h = 0; h < KSUB; ++h) {
               const uint32_t dst = smem_u32(k_tiles + kr.stage * kStageBytes + v * kSlotBytes + h * kSubTileBytes);
               if (a.block_tokens > 0)
-                tma_load_4d_hint(dst, &maps.k[layer], h * 64, key0 % a.block_tokens, hk, tile_block[lt], bars.k_full(kr.stage), policy);
+                tma_load_4d_hint(dst, &maps.k[layer], h * XSUB, key0 % a.block_tokens, hk, tile_block[lt], bars.k_full(kr.stage), policy);
               else
-                tma_load_3d(dst, &maps.k[layer], h * 64, key0, hk, bars.k_full(kr.stage), policy);
+                tma_load_3d(dst, &maps.k[layer], h * XSUB, key0, hk, bars.k_full(kr.stage), policy);
             }
           } else {
             mbar_arrive(bars.k_full(kr.stage));
@@ -622,17 +703,16 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
     // lane issues the tensor-core instructions =====
     {
       Ring kr(a.k_stages), qr(kQStages), tr(a.t_stages);
-      constexpr uint32_t idesc = instr_desc(NCOLS);
-      const uint64_t k_desc0 = smem_desc(smem_u32(k_tiles));
-      const uint64_t q_desc0 = smem_desc(smem_u32(q_tiles));
+      constexpr uint32_t idesc = instr_desc(NCOLS, FP8);
+      const uint64_t k_desc0 = smem_desc<SUBROW>(smem_u32(k_tiles));
+      const uint64_t q_desc0 = smem_desc<SUBROW>(smem_u32(q_tiles));
       bool ok = true;
       for (int t = 0; ok && t < n_slabs + a.lag; ++t) {
         const bool v1 = t < n_slabs && a.mode != 2, v2 = t >= a.lag && a.mode != 1;
         if (!(ok = mbar_wait_warp(bars.q_full(qr.stage), qr.phase, ab))) break;
         const uint64_t bd0 = q_desc0 + (uint64_t)((qr.stage * 2 * kQSlotBytes) >> 4);
         for (int lt = 0; lt < my_tiles; ++lt) {
-          if (!(ok = mbar_wait_warp(bars.k_full(kr.stage), kr.phase, ab))) break;
-          if (!(ok = mbar_wait_warp(bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
+          if (!(ok = mbar_wait2_warp(bars.k_full(kr.stage), kr.phase, bars.t_empty(tr.stage), tr.phase ^ 1u, ab))) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(tr.stage * 2 * NCOLS);
           const uint64_t ad0 = k_desc0 + (uint64_t)((kr.stage * kStageBytes) >> 4);
@@ -640,12 +720,17 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
 #pragma unroll
             for (int v = 0; v < 2; ++v) {
               if (v == 0 ? v1 : v2) {
+                // 8-bit keys: the two query terms accumulate into the same columns
 #pragma unroll
-                for (int h = 0; h < KSUB; ++h) {
+                for (int part = 0; part < QPARTS; ++part) {
 #pragma unroll
-                  for (int ks = 0; ks < 4; ++ks)
-                    tc_mma(d_tmem + (uint32_t)(v * NCOLS), ad0 + (uint64_t)((v * kSlotBytes + h * kSubTileBytes) >> 4) + 2u * ks,
-                           bd0 + (uint64_t)((v * kQSlotBytes + h * kQSub) >> 4) + 2u * ks, idesc, (uint32_t)((h | ks) != 0));
+                  for (int h = 0; h < KSUB; ++h) {
+#pragma unroll
+                    for (int ks = 0; ks < KSTEPS; ++ks)
+                      tc_mma<FP8>(d_tmem + (uint32_t)(v * NCOLS), ad0 + (uint64_t)((v * kSlotBytes + h * kSubTileBytes) >> 4) + 2u * ks,
+                                  bd0 + (uint64_t)((v * kQSlotBytes + (part * KSUB + h) * kQSub) >> 4) + 2u * ks, idesc,
+                                  (uint32_t)((part | h | ks) != 0));
+                  }
                 }
               }
             }
@@ -682,7 +767,7 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
         for (int r = 0; r < 2; ++r) {
           const int row = lane + 32 * r;
           if (row < rows_real)
-            value[r] = __ldg(a.lse_in + ((int64_t)slab * G + row % G) * a.n_lookahead + row / G) * kLog2e * a.inv_c;
+            value[r] = __ldg(a.lse_in + ((int64_t)slab * G + row % G) * a.n_lookahead + row / G) * kLog2e * (FP8 ? 1.f : a.inv_c);
         }
         if (use > 0) {
           if (!(ok = mbar_wait_warp(bars.o_free(x), (uint32_t)(use - 1) & 1u, ab))) break;
@@ -691,6 +776,9 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
         for (int r = 0; r < 2; ++r) {
           const int row = lane + 32 * r;
           if (row < NCOLS) rowoff[x * 64 + row] = value[r];
+        }
+        if constexpr (FP8) {
+          if (lane == 0) slab_c[x] = __ldg(a.slab_scale + slab);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bars.o_ready(x));
@@ -731,7 +819,7 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
           }
           if (!(lse2 > -INFINITY && lse2 < INFINITY) && a.dev_status != nullptr)
             atomicCAS(a.dev_status, 0, (int32_t)SPF_ERR_RANGE);
-          value[r] = lse2 * a.inv_c;                            // lse in q.k units
+          value[r] = FP8 ? lse2 : lse2 * a.inv_c;               // lse in q.k units (8-bit keys: in base-2 logits, the scale differs per slab)
           if (cta == 0 && a.lse_out != nullptr) a.lse_out[out_idx] = lse2 * kLn2;
         }
       }
@@ -743,6 +831,9 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
       for (int r = 0; r < 2; ++r) {
         const int row = lane + 32 * r;
         if (row < NCOLS) rowoff[x * 64 + row] = value[r];
+      }
+      if constexpr (FP8) {
+        if (lane == 0) slab_c[x] = __ldg(a.slab_scale + slab);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bars.o_ready(x));
@@ -769,10 +860,19 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
     constexpr int BATCH = PASSES < 8 ? PASSES : 8;              // loads in flight per lane
     for (int slab = cta; slab < n_slabs && a.mode != 2; slab += n_cta) {
       const int layer = slab / a.n_kv_heads, hk = slab % a.n_kv_heads;
-      const uint4 kv = __ldg(reinterpret_cast<const uint4*>(a.k_layers[layer] + sample_block * a.stride_block + hk * a.stride_head +
-                                                            sample_row * a.stride_tok) + lane % LPR);
       float kf[8];
-      {
+      if constexpr (FP8) {
+        // strides count bytes; a lane's 8 keys elements are 8 bytes
+        const uint2 kv = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned char*>(a.k_layers[layer]) +
+                                                              hk * a.stride_head + sample_row * a.stride_tok) + lane % LPR);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          kf[e] = e4m3_to_float(kv.x >> (8 * e));
+          kf[4 + e] = e4m3_to_float(kv.y >> (8 * e));
+        }
+      } else {
+        const uint4 kv = __ldg(reinterpret_cast<const uint4*>(a.k_layers[layer] + sample_block * a.stride_block + hk * a.stride_head +
+                                                              sample_row * a.stride_tok) + lane % LPR);
         const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&kv);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -808,20 +908,24 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
       }
 #pragma unroll
       for (int off = 16; off >= LPR; off >>= 1) ref = fminf(ref, __shfl_xor_sync(0xffffffffu, ref, off));
-      ref = fmaf(ref, a.c, kRefMargin);                          // base-2 units, plus the margin
+      ref = fmaf(ref, FP8 ? a.c * __ldg(a.key_scale + slab) : a.c, kRefMargin);   // base-2 units, plus the margin
       if (lane == 0) {
         const unsigned word = __float_as_uint(ref) | 1u;
         asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.refs + slab), "r"(word) : "memory");
       }
     }
     unsigned mine = 0u;                                          // lane's reference of slab (slab & ~31) + lane
+    float mine_c = 0.f;                                          // 8-bit keys: and its slab_scale
     for (int slab = 0; ok && slab < n_slabs && a.mode != 2; ++slab) {
       if ((slab & 31) == 0) {
         mine = 1u;
+        if constexpr (FP8) mine_c = slab + lane < n_slabs ? __ldg(a.slab_scale + slab + lane) : 0.f;
         const bool got = slab + lane >= n_slabs || word_wait(a.refs + slab + lane, mine, ab);
         if (!(ok = __all_sync(0xffffffffu, got))) break;
       }
       const float ref = __uint_as_float(__shfl_sync(0xffffffffu, mine, slab & 31));
+      float ref_c = 0.f;
+      if constexpr (FP8) ref_c = __shfl_sync(0xffffffffu, mine_c, slab & 31);
       const int x = slab & 1;
       const int use = slab >> 1;
       if (use > 0) {
@@ -830,6 +934,7 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
       }
       if (lane == 0) {
         rowoff[x * 64] = ref;
+        if constexpr (FP8) slab_c[x] = ref_c;
         ref_slots[slab % kRefSlots] = ref;
         __threadfence_block();
         misc[3] = slab + 1;                                    // the log-sum-exp warp reads ref_slots after this
@@ -876,6 +981,7 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
         const int slab = t, x1 = slab & 1;
         if (!(ok = mbar_wait_warp(bars.o_ready(x1), (uint32_t)(slab >> 1) & 1u, ab))) break;
         const float nref = -rowoff[x1 * 64];                    // one reference per slab
+        const float c1 = FP8 ? slab_c[x1] : a.c;                // accumulated dot product -> base-2 logit
         __syncwarp();
         if (lane == 0) mbar_arrive(bars.o_free(x1));
         float sum[CW];
@@ -904,7 +1010,7 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
             // per-thread sums of exp2 over the thread's keys
             if (real) {
 #pragma unroll
-              for (int j = 0; j < CHK; ++j) sum[c * CHK + j] += fast_exp2(fmaf(__uint_as_float(r[j]), a.c, nref));
+              for (int j = 0; j < CHK; ++j) sum[c * CHK + j] += fast_exp2(fmaf(__uint_as_float(r[j]), c1, nref));
             }
           }
         }
@@ -1002,6 +1108,7 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
         const int slab = t - a.lag, x2 = 2 + (slab & 1);
         if (!(ok = mbar_wait_warp(bars.o_ready(x2), (uint32_t)(slab >> 1) & 1u, ab))) break;
         const float4* off2 = reinterpret_cast<const float4*>(rowoff + x2 * 64 + half * CW);
+        [[maybe_unused]] const float c2 = FP8 ? slab_c[x2] : 0.f;
         for (int lt = 0; lt < my_tiles; ++lt) {
           if (!(ok = mbar_wait_warp(bars.t_full(tr.stage), tr.phase, ab))) break;
           tc_fence_after();
@@ -1035,9 +1142,11 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
             // running max over (layer, head) of q.k - lse/c (slots past n_lookahead hold padding and are never read)
 #pragma unroll
             for (int ii = 0; ii < CHK / G; ++ii) {
-              float mx = __uint_as_float(r[ii * G]) - o[ii * G];
+              // bf16 keys: q.k - lse/c, one scale for all slabs; 8-bit keys: base-2 logit - lse, the scale differs per slab
+              float mx = FP8 ? fmaf(__uint_as_float(r[ii * G]), c2, -o[ii * G]) : __uint_as_float(r[ii * G]) - o[ii * G];
 #pragma unroll
-              for (int g = 1; g < G; ++g) mx = fmaxf(mx, __uint_as_float(r[ii * G + g]) - o[ii * G + g]);
+              for (int g = 1; g < G; ++g)
+                mx = fmaxf(mx, FP8 ? fmaf(__uint_as_float(r[ii * G + g]), c2, -o[ii * G + g]) : __uint_as_float(r[ii * G + g]) - o[ii * G + g]);
               const int i = c * (CHK / G) + ii;
               am[i / AC][i % AC] = __float_as_uint(fmaxf(__uint_as_float(am[i / AC][i % AC]), mx));
             }
@@ -1070,7 +1179,7 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
           tmem_wait<FC>(v);
 #pragma unroll
           for (int j = 0; j < FC; ++j)
-            if (q * FC + j < a.n_lookahead) sacc += fast_exp2(__uint_as_float(v[j]) * a.c);
+            if (q * FC + j < a.n_lookahead) sacc += fast_exp2(FP8 ? __uint_as_float(v[j]) : __uint_as_float(v[j]) * a.c);
         }
         if (key < a.n_tokens) a.importance[key] = sacc * inv_m;
       }
@@ -1089,6 +1198,59 @@ __global__ void __launch_bounds__(SPF_FUSED_LB, 1) score_fused_kernel(const __gr
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- 8-bit keys: query split
+// The tensor cores multiply E4M3 keys only by operands of an 8-bit format, so a slab's bf16 queries are handed over as
+// two E4M3 terms, q * S = hi + lo: hi = the nearest E4M3 of q * S, lo = the nearest E4M3 of the remainder.  S is a power
+// of two per slab that puts the slab's largest |q| just below the format's maximum (448).  A bf16 has 8 significant
+// bits and each term carries 4, so the pair is exact for every element within 2^9 of the slab's largest and off by at
+// most 2^-17 of that largest value below (the remainder's last bits fall under the format's smallest step, 2^-9).  One
+// block per slab writes [slab][term][NCOLS rows][d] bytes (row j = i * G + g, padding rows zero) and the slab's
+// factor from accumulated dot product to base-2 logit: softmax scale * log2(e) * key scale / S.
+__global__ void __launch_bounds__(256) split_q_kernel(const __nv_bfloat16* __restrict__ q, int G, int m, int d, int ncols,
+                                                      const float* __restrict__ key_scale, float c, unsigned char* __restrict__ out,
+                                                      float* __restrict__ slab_scale) {
+  const int slab = blockIdx.x;
+  const int rows = G * m, n = rows * d;
+  __shared__ float red[8];
+  __shared__ float s_scale;
+  float mx = 0.f;
+  for (int idx = threadIdx.x; idx < n; idx += blockDim.x) {
+    const int j = idx / d, e = idx - j * d;
+    mx = fmaxf(mx, fabsf(__bfloat162float(q[(((int64_t)slab * G + j % G) * m + j / G) * d + e])));
+  }
+  for (int off = 16; off >= 1; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
+    // largest power of two S with mx * S <= 448 (mx = 0 or not finite: S = 1)
+    float S = 1.f;
+    if (mx > 0.f && mx < INFINITY) {
+      int ex;
+      const float fr = frexpf(448.f / mx, &ex);   // 448 / mx = fr * 2^ex, fr in [0.5, 1)
+      (void)fr;
+      S = ldexpf(1.f, max(-100, min(ex - 1, 100)));
+    }
+    s_scale = S;
+    slab_scale[slab] = c * key_scale[slab] / S;
+  }
+  __syncthreads();
+  const float S = s_scale;
+  unsigned char* hi = out + (int64_t)slab * 2 * ncols * d;
+  unsigned char* lo = hi + (int64_t)ncols * d;
+  for (int idx = threadIdx.x; idx < ncols * d; idx += blockDim.x) {
+    const int j = idx / d, e = idx - j * d;
+    uint32_t h = 0u, l = 0u;
+    if (j < rows) {
+      const float v = __bfloat162float(q[(((int64_t)slab * G + j % G) * m + j / G) * d + e]) * S;
+      h = float_to_e4m3(v);
+      l = float_to_e4m3(v - e4m3_to_float(h));
+    }
+    hi[idx] = (unsigned char)h;
+    lo[idx] = (unsigned char)l;
   }
 }
 
@@ -1121,7 +1283,14 @@ constexpr int kSmemBudget = 227 * 1024 - 1024;   // dynamic shared memory we may
 FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
   FusedPlan pl;
   const int g = p.group;
-  if (p.k_scale != nullptr) return pl;        // 8-bit key caches: general path only
+  const bool fp8 = p.k_scale != nullptr;
+  // 8-bit key caches: contiguous only, and the TMA wants 16-byte aligned layer pointers and strides (the general path
+  // reads them 8 bytes at a time and takes what this refuses)
+  if (fp8) {
+    if (p.block_tokens > 0 || p.stride_tok % 16 != 0 || p.stride_head % 16 != 0) return pl;
+    for (int l = 0; l < p.n_layers; ++l)
+      if (reinterpret_cast<uintptr_t>(p.k.p[l]) % 16 != 0) return pl;
+  }
   if (!(g == 1 || g == 2 || g == 4 || g == 8)) return pl;
   if (p.n_layers > kFusedMaxLayers) return pl;
   const int rows = g * p.n_lookahead;
@@ -1137,7 +1306,7 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
     if (ts * 2 * pl.ncols + amax_cols <= kTmemColsAll) pl.t_stages = ts;
   if (pl.t_stages == 0) return pl;
   for (int ks = 10; ks >= 2; --ks) {
-    const SmemLayout lay = smem_layout(p.head_dim, pl.ncols, g, ks, pl.tiles_per_cta_max);
+    const SmemLayout lay = smem_layout(p.head_dim, fp8, pl.ncols, g, ks, pl.tiles_per_cta_max);
     if ((int)lay.total <= kSmemBudget) {
       pl.k_stages = ks;
       pl.lay = lay;
@@ -1154,14 +1323,15 @@ FusedPlan make_plan(const ScoreProblem& p, int sm_count) {
 // three slabs of lead at 16 MB a slab (measured at 128k tokens, d = 64: lag 2..4 within 1 %, 5 and 6 cost 6 and 11 %;
 // at 64k tokens, d = 128: lag 3 best, 2 and 4 cost 9 and 3 %, 5 costs 22 %).
 int fused_lag(const ScoreProblem& p, int n_slabs) {
-  const double slab_bytes = (double)p.n_tokens * p.head_dim * 2.0;
+  const double slab_bytes = (double)p.n_tokens * row_bytes(p.head_dim, p.k_scale != nullptr);
   int lag = (int)(64.0 * 1024 * 1024 / slab_bytes) - 1;
   lag = std::max(2, std::min(lag, 8));
   return std::max(1, std::min(lag, n_slabs));
 }
 
 struct FusedWorkspace {
-  size_t limbs_off, counters_off, refs_off, total;   // all three are cleared before every launch
+  size_t limbs_off, counters_off, refs_off, clear_bytes;   // [0, clear_bytes) is cleared before every launch
+  size_t qsplit_off, slab_scale_off, total;               // 8-bit keys: the split queries and the per-slab factors
 };
 
 FusedWorkspace fused_workspace(const ScoreProblem& p) {
@@ -1170,7 +1340,12 @@ FusedWorkspace fused_workspace(const ScoreProblem& p) {
   w.limbs_off = 0;
   w.counters_off = align_up(n_slabs * 64 * kLimbStride * sizeof(unsigned long long), 256);
   w.refs_off = align_up(w.counters_off + n_slabs * sizeof(unsigned), 256);
-  w.total = align_up(w.refs_off + n_slabs * sizeof(unsigned), 256);
+  w.clear_bytes = align_up(w.refs_off + n_slabs * sizeof(unsigned), 256);
+  w.qsplit_off = w.slab_scale_off = w.total = w.clear_bytes;
+  if (p.k_scale != nullptr) {
+    w.slab_scale_off = align_up(w.qsplit_off + n_slabs * 2 * 64 * (size_t)p.head_dim, 256);
+    w.total = align_up(w.slab_scale_off + n_slabs * sizeof(float), 256);
+  }
   return w;
 }
 
@@ -1179,9 +1354,9 @@ FusedWorkspace fused_workspace(const ScoreProblem& p) {
 // co-resident -- fewer SMs available than the device reports, e.g. under MPS with a limited SM share -- is refused
 // here instead of spinning into the bounded waits.  SMs that are merely busy with other kernels delay the launch;
 // they do not break it.
-template <int D, int NCOLS, int G>
+template <int D, int NCOLS, int G, bool FP8>
 int32_t launch_fused(const FusedMaps& maps, const FusedArgs& args, const FusedPlan& pl, cudaStream_t stream) {
-  auto kern = score_fused_kernel<D, NCOLS, G>;
+  auto kern = score_fused_kernel<D, NCOLS, G, FP8>;
   const int smem_bytes = (int)pl.lay.total + 1024;
   SPF_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
   int per_sm = 0;
@@ -1207,26 +1382,26 @@ int32_t launch_fused(const FusedMaps& maps, const FusedArgs& args, const FusedPl
   return SPF_OK;
 }
 
-template <int D, int NCOLS>
+template <int D, int NCOLS, bool FP8>
 int32_t launch_fused_g(int g, const FusedMaps& maps, const FusedArgs& args, const FusedPlan& pl, cudaStream_t stream) {
   // a thread owns NCOLS / 2 query rows, which must hold whole GQA groups
   if constexpr (NCOLS >= 16) {
     switch (g) {
-      case 1: return launch_fused<D, NCOLS, 1>(maps, args, pl, stream);
-      case 2: return launch_fused<D, NCOLS, 2>(maps, args, pl, stream);
-      case 4: return launch_fused<D, NCOLS, 4>(maps, args, pl, stream);
-      default: return launch_fused<D, NCOLS, 8>(maps, args, pl, stream);
+      case 1: return launch_fused<D, NCOLS, 1, FP8>(maps, args, pl, stream);
+      case 2: return launch_fused<D, NCOLS, 2, FP8>(maps, args, pl, stream);
+      case 4: return launch_fused<D, NCOLS, 4, FP8>(maps, args, pl, stream);
+      default: return launch_fused<D, NCOLS, 8, FP8>(maps, args, pl, stream);
     }
   }
   return SPF_ERR_UNSUPPORTED;
 }
 
-template <int D>
+template <int D, bool FP8>
 int32_t launch_fused_n(int ncols, int g, const FusedMaps& maps, const FusedArgs& args, const FusedPlan& pl, cudaStream_t stream) {
   switch (ncols) {
-    case 16: return launch_fused_g<D, 16>(g, maps, args, pl, stream);
-    case 32: return launch_fused_g<D, 32>(g, maps, args, pl, stream);
-    default: return launch_fused_g<D, 64>(g, maps, args, pl, stream);
+    case 16: return launch_fused_g<D, 16, FP8>(g, maps, args, pl, stream);
+    case 32: return launch_fused_g<D, 32, FP8>(g, maps, args, pl, stream);
+    default: return launch_fused_g<D, 64, FP8>(g, maps, args, pl, stream);
   }
 }
 
@@ -1270,7 +1445,20 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   FusedMaps maps;
   const int d = p.head_dim, g = p.group, m = p.n_lookahead;
   const int n_slabs = p.n_layers * p.n_kv_heads;
-  {
+  const bool fp8 = p.k_scale != nullptr;
+  const int subrow = sub_row_bytes(row_bytes(d, fp8));
+  const CUtensorMapSwizzle swizzle = subrow == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+  if (fp8) {
+    // (d, row, slab * 2 + term) view of the split queries, which split_q_kernel writes below
+    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)pl.ncols, (cuuint64_t)n_slabs * 2};
+    const cuuint64_t strides[2] = {(cuuint64_t)d, (cuuint64_t)pl.ncols * d};
+    const cuuint32_t box[3] = {(cuuint32_t)subrow, (cuuint32_t)pl.ncols, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = encode(&maps.q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, base + w.qsplit_off, dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(SPF_ERR_CUDA, "spf_score_fp8: encoding the query tensor map failed (CUresult %d)", (int)r);
+  } else {
     const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)g, (cuuint64_t)m, (cuuint64_t)n_slabs};
     const cuuint64_t strides[3] = {(cuuint64_t)m * d * 2, (cuuint64_t)d * 2, (cuuint64_t)g * m * d * 2};
     const cuuint32_t box[4] = {64, (cuuint32_t)g, (cuuint32_t)m, 1};
@@ -1293,7 +1481,20 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
     if (r != CUDA_SUCCESS)
       return fail(SPF_ERR_CUDA, "spf_score_paged: encoding the key tensor map of layer %d failed (CUresult %d)", l, (int)r);
   }
-  for (int l = 0; l < p.n_layers && p.block_tokens == 0; ++l) {
+  for (int l = 0; l < p.n_layers && fp8; ++l) {
+    // 8-bit keys: strides count bytes
+    const cuuint64_t head_stride = p.n_kv_heads > 1 ? (cuuint64_t)p.stride_head : (cuuint64_t)p.stride_tok * p.n_tokens;
+    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)p.n_tokens, (cuuint64_t)p.n_kv_heads};
+    const cuuint64_t strides[2] = {(cuuint64_t)p.stride_tok, head_stride};
+    const cuuint32_t box[3] = {(cuuint32_t)subrow, (cuuint32_t)kTileKeys, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = encode(&maps.k[l], CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<__nv_bfloat16*>(p.k.p[l]), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+      return fail(SPF_ERR_CUDA, "spf_score_fp8: encoding the key tensor map of layer %d failed (CUresult %d)", l, (int)r);
+  }
+  for (int l = 0; l < p.n_layers && p.block_tokens == 0 && !fp8; ++l) {
     const cuuint64_t head_stride = p.n_kv_heads > 1 ? (cuuint64_t)p.stride_head : (cuuint64_t)p.stride_tok * p.n_tokens;
     const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)p.n_tokens, (cuuint64_t)p.n_kv_heads};
     const cuuint64_t strides[2] = {(cuuint64_t)p.stride_tok * 2, head_stride * 2};
@@ -1327,6 +1528,8 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   args.limbs = reinterpret_cast<unsigned long long*>(base + w.limbs_off);
   args.counters = reinterpret_cast<unsigned*>(base + w.counters_off);
   args.refs = reinterpret_cast<unsigned*>(base + w.refs_off);
+  args.slab_scale = fp8 ? reinterpret_cast<const float*>(base + w.slab_scale_off) : nullptr;
+  args.key_scale = p.k_scale;
   args.lse_out = p.lse_out;
   args.extra_lse = p.extra_lse;
   args.importance = p.importance;
@@ -1336,9 +1539,17 @@ int32_t score_fused_launch(const ScoreProblem& p, void* workspace, int sm_count,
   args.stride_block = (int64_t)p.n_kv_heads * p.block_tokens * p.head_dim;
   args.n_pool_blocks = p.n_pool_blocks;
 
-  SPF_CUDA_CHECK(cudaMemsetAsync(base, 0, w.total, stream));
-  if (d == 64) return launch_fused_n<64>(pl.ncols, g, maps, args, pl, stream);
-  return launch_fused_n<128>(pl.ncols, g, maps, args, pl, stream);
+  SPF_CUDA_CHECK(cudaMemsetAsync(base, 0, w.clear_bytes, stream));
+  if (fp8) {
+    split_q_kernel<<<n_slabs, 256, 0, stream>>>(p.q, g, m, d, pl.ncols, p.k_scale, p.c_log2,
+                                                reinterpret_cast<unsigned char*>(base + w.qsplit_off),
+                                                reinterpret_cast<float*>(base + w.slab_scale_off));
+    SPF_CUDA_CHECK(cudaGetLastError());
+    if (d == 64) return launch_fused_n<64, true>(pl.ncols, g, maps, args, pl, stream);
+    return launch_fused_n<128, true>(pl.ncols, g, maps, args, pl, stream);
+  }
+  if (d == 64) return launch_fused_n<64, false>(pl.ncols, g, maps, args, pl, stream);
+  return launch_fused_n<128, false>(pl.ncols, g, maps, args, pl, stream);
 }
 
 }  // namespace spf

@@ -1,5 +1,7 @@
-"""8-bit key caches (spf_score_fp8) against the oracle on the same bytes: small shapes with ragged tails, every
-row-count template of the general kernels, strided caches, and the long-context geometry at full size."""
+"""8-bit key caches (spf_score_fp8) against the oracle on the same bytes, on both kernel paths: small shapes with ragged
+tails, every row-count template, strided caches, and the long-context geometry at full size.  The fused path feeds the
+tensor cores E4M3 keys and queries split into two E4M3 terms (exact but for elements 2^9 below a slab's largest), so
+the same tolerances hold on both paths."""
 import numpy as np
 import pytest
 import torch
@@ -25,18 +27,29 @@ SHAPES = [
 ]
 
 
+@pytest.fixture(params=["general", "fused"])
+def kernel_path(request):
+    """Pins the scoring path for one test; a shape the fused path refuses (status -2) turns into a skip (conftest)."""
+    import paper_2603_02631_b200 as spf
+    previous = spf.spf_set_score_path(1 if request.param == "general" else 2)
+    yield request.param
+    spf.spf_set_score_path(previous)
+
+
 def _run(spf, q, k8, scales, n, lse_rows):
     imp = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
     lse = torch.full((lse_rows,), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
     bufs = spf.Fp8PromptBuffers(q, k8, scales, imp, lse)
     ws = torch.empty(spf.spf_score_fp8_workspace_bytes([bufs]), dtype=torch.uint8, device="cuda")
-    spf.spf_score_fp8([bufs], ws)
+    spf.spf_score_fp8([bufs], ws, 0.0, status)
     torch.cuda.synchronize()
+    assert int(status.item()) == 0
     return imp.cpu().numpy(), lse.cpu().numpy()
 
 
 @pytest.mark.parametrize("L,Hq,Hkv,d,m,N", SHAPES)
-def test_fp8_small_shapes(L, Hq, Hkv, d, m, N):
+def test_fp8_small_shapes(kernel_path, L, Hq, Hkv, d, m, N):
     import paper_2603_02631_b200 as spf
     cfg = small_config("fp8", n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, n_lookahead=m, lengths=(N,),
                        rank=4, n_needles=2 if N >= 300 else 0, n_strong=1, needle_len=(4, 40), seed=N + m)
@@ -48,7 +61,7 @@ def test_fp8_small_shapes(L, Hq, Hkv, d, m, N):
     np.testing.assert_allclose(got_lse.reshape(want_lse.shape), want_lse, rtol=0, atol=2e-4)
 
 
-def test_fp8_every_byte_value_is_decoded_exactly():
+def test_fp8_every_byte_value_is_decoded_exactly(kernel_path):
     """A cache that holds every finite E4M3 byte: one head, d = 64, query = a unit vector along each coordinate in turn, so
     each logit is one decoded key value times the scale (exact in fp32): checks the kernel's decoder bit for bit through
     the log-sum-exp and the importance."""
@@ -69,22 +82,24 @@ def test_fp8_every_byte_value_is_decoded_exactly():
     np.testing.assert_allclose(got_lse.reshape(want_lse.shape), want_lse, rtol=0, atol=2e-4)
 
 
-def test_fp8_strided_cache():
-    """Keys interleaved with other data (a fused KV layout): strides in bytes, rows 8-byte aligned."""
+@pytest.mark.parametrize("row,first", [(136, 8), (144, 16)])
+def test_fp8_strided_cache(kernel_path, row, first):
+    """Keys interleaved with other data (a fused KV layout): strides in bytes.  Rows 8-byte aligned are enough for the
+    general path; the fused path wants 16 (and refuses the other case, which the automatic choice hands to the general path)."""
     import paper_2603_02631_b200 as spf
     cfg = small_config("fp8s", n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, n_lookahead=8, lengths=(777,), rank=4, seed=9)
     prompt = make_prompt(cfg)
     k8, scales = quantize_keys_e4m3(prompt.k)
-    wide = [torch.full((2, 777, 136), 0x7E, dtype=torch.uint8, device="cuda") for _ in k8]   # 448s around the keys
+    wide = [torch.full((2, 777, row), 0x7E, dtype=torch.uint8, device="cuda") for _ in k8]   # 448s around the keys
     for w, x in zip(wide, k8):
-        w[:, :, 8:72] = x.cuda()
-    views = [w[:, :, 8:72] for w in wide]
+        w[:, :, first:first + 64] = x.cuda()
+    views = [w[:, :, first:first + 64] for w in wide]
     want, _ = oracle.token_importance_fp8(bf16_bits(prompt.q), [x.numpy() for x in k8], scales.numpy())
     got, _ = _run(spf, prompt.q.cuda(), views, scales.cuda(), 777, 2 * 4 * 8)
     assert_importance_close(got, want)
 
 
-def test_fp8_long_context_full_size():
+def test_fp8_long_context_full_size(kernel_path):
     """The long-context configuration with its key cache in 8 bits, end to end (score -> pool -> top-k -> spans)."""
     import paper_2603_02631_b200 as spf
     cfg = CONFIGS["long128k"]
@@ -110,15 +125,32 @@ def test_fp8_long_context_full_size():
                                        char_spans=o_ch), prompt)
 
 
-def test_fp8_is_refused_on_the_forced_fused_path():
+def test_fp8_queries_with_a_wide_dynamic_range(kernel_path):
+    """Query elements spread over 2^-14 .. 1 of their slab's largest: on the fused path the small ones pass the two-term
+    split inexactly (by at most 2^-17 of the largest), which must stay far inside the tolerance."""
     import paper_2603_02631_b200 as spf
-    cfg = small_config("fp8r", n_layers=1, n_q_heads=2, n_kv_heads=1, head_dim=64, n_lookahead=8, lengths=(300,), seed=1)
+    cfg = small_config("fp8w", n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=64, n_lookahead=8, lengths=(1500,), rank=4,
+                       n_needles=2, n_strong=1, needle_len=(4, 40), seed=77)
+    prompt = make_prompt(cfg)
+    g = torch.Generator().manual_seed(5)
+    expo = torch.randint(-14, 1, prompt.q.shape, generator=g).to(torch.float32)
+    q = (prompt.q.to(torch.float32) * torch.exp2(expo) * 8.0).to(torch.bfloat16)
+    k8, scales = quantize_keys_e4m3(prompt.k)
+    want, want_lse = oracle.token_importance_fp8(bf16_bits(q), [x.numpy() for x in k8], scales.numpy())
+    got, got_lse = _run(spf, q.cuda(), [x.cuda() for x in k8], scales.cuda(), 1500, 2 * 8 * 8)
+    assert_importance_close(got, want)
+    np.testing.assert_allclose(got_lse.reshape(want_lse.shape), want_lse, rtol=0, atol=2e-4)
+
+
+def test_fp8_unaligned_cache_goes_to_the_general_path_by_itself():
+    """Rows that start 8 bytes into a 16-byte unit: the fused path cannot read them, the automatic choice must not try."""
+    import paper_2603_02631_b200 as spf
+    cfg = small_config("fp8u", n_layers=1, n_q_heads=2, n_kv_heads=1, head_dim=64, n_lookahead=8, lengths=(300,), seed=1)
     prompt = make_prompt(cfg)
     k8, scales = quantize_keys_e4m3(prompt.k)
-    previous = spf.spf_set_score_path(2)
-    try:
-        with pytest.raises(spf.SpfError) as err:
-            _run(spf, prompt.q.cuda(), [x.cuda() for x in k8], scales.cuda(), 300, 2 * 8)
-        assert err.value.status == -2
-    finally:
-        spf.spf_set_score_path(previous)
+    wide = torch.zeros((1, 300, 136), dtype=torch.uint8, device="cuda")
+    wide[:, :, 8:72] = k8[0].cuda()
+    want, _ = oracle.token_importance_fp8(bf16_bits(prompt.q), [k8[0].numpy()], scales.numpy())
+    assert spf.spf_set_score_path(0) == 0
+    got, _ = _run(spf, prompt.q.cuda(), [wide[:, :, 8:72]], scales.cuda(), 300, 2 * 8)
+    assert_importance_close(got, want)

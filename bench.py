@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM read + write bytes of one scoring launch, from the ncu capture summarised in profiles/.  Each entry names
 # the SHA-256 of the kernel source it was taken from: once the source changes, the figure is reported as null.
 NCU_TRAFFIC = {
-    ("long128k", "fused"): {"bytes": 4 * (538848256 + 6746368), "source": "paper_2603_02631_b200/csrc/score_fused.cu",
-                            "sha256": "f5290961f9ccc5026dd9969a7690aeee6bf7d11599bb3aa4194f6eb22d7552f7",
+    ("long128k", "fused"): {"bytes": 4 * (538341120 + 6759680), "source": "paper_2603_02631_b200/csrc/score_fused.cu",
+                            "sha256": "97f49fa8be69ccf6ba8df7c7e8e1053a340d517c09eb1a11f3c31d6407593490",
                             "note": "captured on long128k_l4 (4 of 16 layers), scaled x4"},
 }
 

@@ -647,10 +647,79 @@ def run_keys(args, ops=None, device=None, backend="nccl", cfg=None):
     return line
 
 
+def run_fp8_line(args):
+    """`--workload <name>_fp8`: the whole path on one prompt of <name> whose key cache is held as E4M3 bytes
+    (Selector.run_fp8: spf_score_fp8 -> spf_chunk_pool -> spf_select_compact), device-resident, one GPU.  The roofline's
+    bytes are this format's own: the 8-bit cache read once + scales + Q + importance + lse."""
+    import torch
+    import paper_2603_02631_b200 as spf
+    from workloads import CONFIGS, make_prompt, quantize_keys_e4m3
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    cfg = CONFIGS[args.workload[:-len("_fp8")]]
+    keep = cfg.keep[0]
+    prompt = make_prompt(cfg, 0, dev)
+    k8, scales = quantize_keys_e4m3(prompt.k)
+    q, ids, cs, ce, n = prompt.q, prompt.token_ids, prompt.char_start, prompt.char_end, prompt.n_tokens
+    del prompt
+    torch.cuda.empty_cache()
+    sel = spf.Selector(cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_lookahead, n, chunk=cfg.chunk,
+                       pool_kernel=cfg.pool_kernel, device=dev)
+    spf.spf_set_score_path({"auto": 0, "general": 1, "fused": 2}[args.score_path])
+    stream = torch.cuda.current_stream()
+    for _ in range(max(args.warmup, 3)):
+        sel.run_fp8(q, k8, scales, ids, cs, ce, keep)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    m0 = sampler.mark()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(args.steps):
+        sel.run_fp8(q, k8, scales, ids, cs, ce, keep)
+    b.record(stream)
+    torch.cuda.synchronize()
+    ms_step = a.elapsed_time(b) / args.steps
+    bufs = spf.Fp8PromptBuffers(q, k8, scales, sel.importance[:n], sel.lse)
+    a.record(stream)
+    for _ in range(args.steps):
+        spf.spf_score_fp8([bufs], sel.workspace, 0.0, sel.dev_status)
+    b.record(stream)
+    torch.cuda.synchronize()
+    m1 = sampler.mark()
+    sampler.stop()
+    clocks = sampler.stats(m0, m1)
+    sampler.close()
+    status = int(sel.dev_status.item())
+    if status != 0:
+        raise RuntimeError(f"device status {status} ({spf.spf_status_string(status)})")
+    ms_score = a.elapsed_time(b) / args.steps
+    rows = cfg.n_layers * cfg.n_q_heads * cfg.n_lookahead
+    nbytes = cfg.k_bytes() // 2 + 4 * cfg.n_layers * cfg.n_kv_heads + rows * cfg.head_dim * 2 + 4 * n + 4 * rows
+    peak, peak_kind = hbm_peak()
+    gbs = nbytes / (ms_score * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": n / (ms_step * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "e4m3 keys, two-term e4m3 queries (bf16 in), f32 accumulate/softmax", "data": "synthetic",
+        "config": {"workload": args.workload, "n_tokens": [n], "n_layers": cfg.n_layers, "n_q_heads": cfg.n_q_heads,
+                   "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim, "n_lookahead": cfg.n_lookahead, "chunk": cfg.chunk,
+                   "keep": keep, "k_cache_bytes": cfg.k_bytes() // 2, "score_path": args.score_path,
+                   "l2": "inputs larger than L2 (key cache streamed every step)"},
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "gpu_launches": 4 * args.steps, "e2e": None,
+        "roofline": {"bound": "hbm", "kernel": "spf_score_fp8", "achieved": gbs, "peak": peak, "peak_kind": f"of {peak_kind}",
+                     "unit": "GB/s", "frac": gbs / peak, "traffic": None, "ms_per_launch": ms_score, "algorithmic_bytes": nbytes},
+    }), flush=True)
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload.endswith("_fp8"):
+        run_fp8_line(args)
     elif args.parallelism == "keys":
         run_keys(args)
     else:
